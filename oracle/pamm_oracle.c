@@ -1,0 +1,203 @@
+/*
+ * PAMM oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, fp64 CPU statement of what Point-Approximate Matrix
+ * Multiplication computes for one linear layer (Algorithm 1 "Compress" and
+ * "ApproxMM", Section 3.2, Eq. 1 and Eq. 3 of the paper), at the paper's chosen
+ * setting epsilon -> infinity (Section 4.1: no neighbourhood mask, beta = 1).
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg may call
+ * it.  It shares no code, header, table or constant with the CUDA library.
+ *
+ * Every sum runs in ascending index order in double precision.  OpenMP is used
+ * only across independent outputs (rows of A, columns of B~ / O~); no single
+ * sum is split or reordered.  Inputs arrive in the storage type the GPU gets
+ * (fp32, or bf16 as raw 16-bit patterns) and are widened exactly to double.
+ *
+ * Readings where the paper is silent or inconsistent:
+ *   - Algorithm 1 writes argmax(csim) without the absolute value; Lemma 1 (the
+ *     proven statement) has |csim|.  The oracle follows Lemma 1.
+ *   - The score used is |<A_i,C_j>| / ||C_j||, i.e. |csim| * ||A_i||: the factor
+ *     ||A_i|| is constant per row and does not move the argmax.
+ *   - Ties: the lowest generator index wins.
+ *   - A zero generator (||C_j|| = 0) scores 0 and yields alpha = 0; a zero row
+ *     A_i therefore gets f = 0, alpha = 0.
+ *   - Generator sampling is not done here: the index set I is an input.
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force point-to-line distance argmin
+ * (definition of f below Eq. 1), 1-D line search for alpha, self-representation
+ * alpha = 1, orthogonality of the residual, the factorisation C^T B~ = A~^T B
+ * with A~ from Eq. 3, k = b identity case equal to the exact A^T B, rank-1 A,
+ * the Frobenius error bound of Section 3.2.1, and the printed gamma ~ 28.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+
+static double widen(const void *base, int dtype, int64_t idx)
+{
+    if (dtype == ORACLE_F32) {
+        return (double)((const float *)base)[idx];
+    } else {
+        uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+        float v;
+        memcpy(&v, &bits, sizeof v);
+        return (double)v;
+    }
+}
+
+/* Algorithm 1, "C <- A[I,:]" and the squared row norms of C.
+ * C_out is k x n doubles, q_out[j] = sum_l C_jl^2. */
+int pamm_oracle_gather(const void *A, int dtype, int64_t b, int64_t n, int64_t lda,
+                       const int32_t *I, int64_t k, double *C_out, double *q_out)
+{
+    for (int64_t j = 0; j < k; ++j) {
+        if (I[j] < 0 || I[j] >= b) return 1;
+        double q = 0.0;
+        for (int64_t l = 0; l < n; ++l) {
+            double c = widen(A, dtype, (int64_t)I[j] * lda + l);
+            C_out[j * n + l] = c;
+            q += c * c;
+        }
+        q_out[j] = q;
+    }
+    return 0;
+}
+
+/* Scores of one row against every generator:
+ *   s_j = <A_i, C_j>,  score_j = |s_j| / sqrt(q_j)   (0 when q_j = 0),
+ *   abssum_j = sum_l |A_il * C_jl|  (for rounding-bound reports in tests). */
+void pamm_oracle_row_scores(const void *A, int dtype, int64_t n, int64_t lda, int64_t i,
+                            const double *C, const double *q, int64_t k,
+                            double *s_out, double *score_out, double *abssum_out)
+{
+    for (int64_t j = 0; j < k; ++j) {
+        double s = 0.0, as = 0.0;
+        for (int64_t l = 0; l < n; ++l) {
+            double p = widen(A, dtype, i * lda + l) * C[j * n + l];
+            s += p;
+            as += fabs(p);
+        }
+        s_out[j] = s;
+        score_out[j] = (q[j] > 0.0) ? fabs(s) / sqrt(q[j]) : 0.0;
+        if (abssum_out) abssum_out[j] = as;
+    }
+}
+
+/* Algorithm 1 "Compress" with epsilon = infinity, given the index set I.
+ *   f_i     = lowest j maximising |<A_i,C_j>| / ||C_j||          (Lemma 1)
+ *   alpha_i = <A_i, C_f> / ||C_f||^2                              (Eq. 1)
+ * Also returns the winning score and the best score among the other
+ * generators (top2 = 0 when k = 1) so that near-ties can be reported. */
+int pamm_oracle_compress(const void *A, int dtype, int64_t b, int64_t n, int64_t lda,
+                         const double *C, const double *q, int64_t k,
+                         int32_t *f_out, double *alpha_out, double *top1_out, double *top2_out)
+{
+    int64_t i;
+#pragma omp parallel for schedule(static)
+    for (i = 0; i < b; ++i) {
+        double best = -1.0, second = 0.0, s_best = 0.0;
+        int64_t jbest = 0;
+        for (int64_t j = 0; j < k; ++j) {
+            double s = 0.0;
+            for (int64_t l = 0; l < n; ++l)
+                s += widen(A, dtype, i * lda + l) * C[j * n + l];
+            double score = (q[j] > 0.0) ? fabs(s) / sqrt(q[j]) : 0.0;
+            if (score > best) {            /* strict: lowest j keeps a tie */
+                if (j > 0) second = best;
+                best = score;
+                s_best = s;
+                jbest = j;
+            } else if (score > second) {
+                second = score;
+            }
+        }
+        f_out[i] = (int32_t)jbest;
+        alpha_out[i] = (q[jbest] > 0.0) ? s_best / q[jbest] : 0.0;
+        if (top1_out) top1_out[i] = best;
+        if (top2_out) top2_out[i] = second;
+    }
+    return 0;
+}
+
+/* Algorithm 1 "ApproxMM", first two steps: B' = alpha (.) B and
+ * B~ <- index_add(B~, 0, f, B'), i.e. B~[j,:] = sum_{i: f_i = j} alpha_i B_i
+ * (Section 3.2, "Approximate Matrix Multiplication"). Rows visited in
+ * ascending i. Bt_out is k x m doubles. */
+int pamm_oracle_contract(const int32_t *f, const double *alpha, const void *B, int dtype,
+                         int64_t b, int64_t m, int64_t ldb, int64_t k, double *Bt_out)
+{
+    for (int64_t i = 0; i < b; ++i)
+        if (f[i] < 0 || f[i] >= k) return 1;
+    int64_t c;
+#pragma omp parallel for schedule(static)
+    for (c = 0; c < m; ++c) {
+        for (int64_t j = 0; j < k; ++j) Bt_out[j * m + c] = 0.0;
+        for (int64_t i = 0; i < b; ++i)
+            Bt_out[(int64_t)f[i] * m + c] += alpha[i] * widen(B, dtype, i * ldb + c);
+    }
+    return 0;
+}
+
+/* Algorithm 1 "ApproxMM", last step: O~ = C^T B~ = sum_j C_j^T B~_j  (n x m). */
+void pamm_oracle_weight_grad(const double *C, const double *Bt, int64_t k, int64_t n, int64_t m,
+                             double *O_out)
+{
+    int64_t r;
+#pragma omp parallel for schedule(static)
+    for (r = 0; r < n; ++r) {
+        for (int64_t c = 0; c < m; ++c) {
+            double acc = 0.0;
+            for (int64_t j = 0; j < k; ++j) acc += C[j * n + r] * Bt[j * m + c];
+            O_out[r * m + c] = acc;
+        }
+    }
+}
+
+/* Eq. 3 with every row kept: A~_i = alpha_i * C_{f(i)}  (b x n). */
+void pamm_oracle_reconstruct(const double *C, const int32_t *f, const double *alpha,
+                             int64_t b, int64_t n, double *At_out)
+{
+    for (int64_t i = 0; i < b; ++i)
+        for (int64_t l = 0; l < n; ++l)
+            At_out[i * n + l] = alpha[i] * C[(int64_t)f[i] * n + l];
+}
+
+/* The exact product the method approximates: O = A^T B (Section 3.2), a plain
+ * triple loop; used only on reduced sizes. */
+void pamm_oracle_exact_product(const void *A, int dtypeA, int64_t lda, const void *B, int dtypeB,
+                               int64_t ldb, int64_t b, int64_t n, int64_t m, double *O_out)
+{
+    int64_t r;
+#pragma omp parallel for schedule(static)
+    for (r = 0; r < n; ++r) {
+        for (int64_t c = 0; c < m; ++c) {
+            double acc = 0.0;
+            for (int64_t i = 0; i < b; ++i)
+                acc += widen(A, dtypeA, i * lda + r) * widen(B, dtypeB, i * ldb + c);
+            O_out[r * m + c] = acc;
+        }
+    }
+}
+
+/* Appendix "Complexity Analysis": scalars stored, k*n + 2*b instead of b*n. */
+int64_t pamm_oracle_memory_scalars(int64_t b, int64_t n, int64_t k) { return k * n + 2 * b; }
+
+/* Appendix "Complexity Analysis": gamma = b*m / (k*(b+m)). */
+double pamm_oracle_gamma(int64_t b, int64_t m, int64_t k)
+{
+    return ((double)b * (double)m) / ((double)k * ((double)b + (double)m));
+}
+
+int pamm_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
