@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the PAMM hot path on B200: tokens/s per fused Q|K|V layer.
+
+One "step" = one pass of the whole path over one batch of synthetic input:
+select generators + compress X (forward), then contract dY + C^T B~ (backward).
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on
+a bounded sample of the same workload instead.
+
+Multi-GPU (torchrun, one rank per GPU) is data-parallel replicas, as in the
+paper's DDP runs: every rank compresses its own tokens with its own generators;
+there is no collective on the data path, only the barrier and the max-over-ranks
+reduction of the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "PAMM compress + weight-grad tokens/sec per QKV layer; achieved HBM GB/s vs peak"
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
+# summarised under profiles/, keyed by workload; None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def dist_setup(n_gpus: int, backend: str):
+    """Initialise torch.distributed when launched with WORLD_SIZE > 1."""
+    import torch.distributed as dist
+    world = env_int("WORLD_SIZE", 1)
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group(backend=backend, rank=env_int("RANK", 0), world_size=world)
+    return env_int("RANK", 0), world
+
+
+def aggregate(ms_local: float, tokens_local: int, device="cpu"):
+    """(max over ranks of the time, sum over ranks of the tokens); identity on one rank."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, tokens_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([tokens_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1]))
+                smax = float(p[2])
+            except ValueError:
+                continue
+            for nm, v in zip(names, p[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            d = json.loads(p.read_text())
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(b, n, m, k, e):
+    """Bytes the method itself must move per step (per layer), by stage."""
+    return {
+        "compress": b * n * e + 8 * b + k * n * e,
+        "contract": b * m * e + 8 * b,
+        "weight_grad": n * m * 4 + k * n * e + k * m * 4,
+    }
+
+
+def run_reference(args):
+    """The fp64 oracle on host cores, on a bounded sample of the workload."""
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return
+    from oracle import pamm_oracle as orc
+    from paper_2506_02939_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    k = w.ks[0]
+    seqs = max(1, min(w.num_seqs, args.ref_tokens // w.seq_len))
+    inp = synth.make_inputs(args.workload, num_seqs=seqs)
+    b = inp.b
+    rng = np.random.default_rng(w.index_seed)
+    I = np.sort(rng.choice(b, size=min(k, b), replace=False)).astype(np.int32)
+
+    def step():
+        orc.pamm(inp.X, I, inp.dY)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    val = b * args.steps / dt
+    sample = f"first {b} of {w.b} tokens of workload {w.name} per step, k={len(I)}, all stages, fp64"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: b={w.b} n={w.n} m={w.m} k={k} {w.dtype}", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_cuda(args):
+    import torch
+    from paper_2506_02939_b200 import build as pamm_build, synth
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the PAMM path has no CPU fallback")
+    local = env_int("LOCAL_RANK", 0)
+    torch.cuda.set_device(local)
+    rank, world = dist_setup(args.gpus, "nccl")
+    if rank == 0:
+        pamm_build.build()
+    barrier()
+    from paper_2506_02939_b200 import pamm
+
+    w = synth.WORKLOADS[args.workload]
+    k = args.k or w.ks[0]
+    e = 2 if w.dtype == "bf16" else 4
+    dt_code = pamm.BF16 if w.dtype == "bf16" else pamm.F32
+    inp = synth.make_inputs(args.workload, seed=w.seed + 7919 * rank)
+    b, n, m = inp.b, w.n, w.m
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+
+    def host_tensor(a):
+        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return t.pin_memory()
+
+    Xh, dYh = host_tensor(inp.X), host_tensor(inp.dY)
+    X, dY = Xh.cuda(non_blocking=True), dYh.cuda(non_blocking=True)
+    dev = X.device
+    idx = torch.empty(k, dtype=torch.int32, device=dev)
+    C = torch.empty((k, n), dtype=tdt, device=dev)
+    invn = torch.empty(2 * k, dtype=torch.float32, device=dev)
+    f = torch.empty(b, dtype=torch.int32, device=dev)
+    alpha = torch.empty(b, dtype=torch.float32, device=dev)
+    Bt = torch.empty((k, m), dtype=torch.float32, device=dev)
+    dW = torch.empty((n, m), dtype=torch.float32, device=dev)
+    ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, dt_code, dev)
+    stream = torch.cuda.current_stream()
+
+    def step(seed):
+        pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+        pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+
+    for s in range(args.warmup):
+        step(w.index_seed + s)
+    torch.cuda.synchronize()
+    status = pamm.last_device_status()
+    if status != pamm.OK:
+        raise SystemExit(f"device status after warm-up: {pamm.status_string(status)}")
+
+    # ---- timed region: device-resident inputs ----------------------------------
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    kev = {kind: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+           for kind in (pamm.PROF_COMPRESS, pamm.PROF_CONTRACT, pamm.PROF_WEIGHT_GRAD)}
+    for kind in kev:                       # create the underlying CUDA events
+        for a, z in kev[kind]:
+            a.record(stream)
+            z.record(stream)
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    launches0 = pamm.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_begin.record(stream)
+    for s in range(K):
+        for kind in kev:
+            pamm.set_profile_events(kind, kev[kind][s][0], kev[kind][s][1])
+        ev[s][0].record(stream)
+        pamm.compress_fused(X, k, w.index_seed + s, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+        ev[s][1].record(stream)
+        pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+        ev[s][2].record(stream)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    for kind in kev:
+        pamm.set_profile_events(kind, None, None)
+    launches = pamm.launch_count() - launches0
+    status = pamm.last_device_status()
+    if status != pamm.OK:
+        raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
+    ms_total_local = t_begin.elapsed_time(t_end)
+    ms_total, tokens = aggregate(ms_total_local, b * K, device=dev)
+    fwd = np.array([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)])
+    bwd = np.array([ev[s][1].elapsed_time(ev[s][2]) for s in range(K)])
+    kern = {kind: np.array([a.elapsed_time(z) for a, z in kev[kind]]) for kind in kev}
+
+    # ---- end to end through the host-buffer entry point ----------------------------
+    arena = pamm.alloc_workspace(pamm.WS_STEP_HOST, b, n, m, k, dt_code, dev)
+    dWh = torch.empty((n, m), dtype=torch.float32).pin_memory()
+    Ke = max(3, min(K, args.e2e_steps))
+    for s in range(2):
+        pamm.qkv_step_host(Xh, dYh, k, w.index_seed + s, dWh, arena, stream=stream)
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for s in range(Ke):
+        pamm.qkv_step_host(Xh, dYh, k, w.index_seed + s, dWh, arena, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    ms_e2e, tokens_e2e = aggregate(e0.elapsed_time(e1), b * Ke, device=dev)
+    checksum = float(dWh.double().abs().sum())
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peaks()
+    ab = algorithmic_bytes(b, n, m, k, e)
+    t_contract = float(kern[pamm.PROF_CONTRACT].mean()) * 1e-3
+    achieved = ab["contract"] / t_contract / 1e9
+    stages = {
+        "compress_ms": float(np.median(fwd)), "contract_wgrad_ms": float(np.median(bwd)),
+        "compress_tokens_per_s": b / (float(np.median(fwd)) * 1e-3),
+        "contract_wgrad_tokens_per_s": b / (float(np.median(bwd)) * 1e-3),
+        "compress_stage_gbs": (ab["compress"]) / (float(np.median(fwd)) * 1e-3) / 1e9,
+        "contract_wgrad_stage_gbs": (ab["contract"] + ab["weight_grad"]) / (float(np.median(bwd)) * 1e-3) / 1e9,
+        "kernel_ms": {"compress": float(kern[pamm.PROF_COMPRESS].mean()), "contract_main": float(kern[pamm.PROF_CONTRACT].mean()),
+                      "weight_grad": float(kern[pamm.PROF_WEIGHT_GRAD].mean())},
+        "kernel_gbs": {"compress": ab["compress"] / (float(kern[pamm.PROF_COMPRESS].mean()) * 1e-3) / 1e9,
+                       "contract_main": achieved,
+                       "weight_grad": ab["weight_grad"] / (float(kern[pamm.PROF_WEIGHT_GRAD].mean()) * 1e-3) / 1e9},
+    }
+    stages["compress_stage_frac"] = stages["compress_stage_gbs"] / peak
+    stages["contract_wgrad_stage_frac"] = stages["contract_wgrad_stage_gbs"] / peak
+    saved = pamm.saved_bytes(b, n, k, dt_code)
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import pamm_oracle as orc
+        seqs = max(1, min(w.num_seqs, args.ref_tokens // w.seq_len))
+        bs = seqs * w.seq_len
+        Xs, dYs = inp.X[:bs], inp.dY[:bs]
+        I = pamm.draw_indices_host(bs, min(k, bs), w.index_seed).numpy()
+        t0 = time.perf_counter()
+        reps = 0
+        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+            orc.pamm(Xs, I, dYs)
+            reps += 1
+        dt = time.perf_counter() - t0
+        cpu = {"value": bs * reps / dt, "unit": "tokens/s", "cores": orc.num_threads(), "kind": "oracle",
+               "sample": f"first {bs} of {b} tokens, k={min(k, bs)}, all stages, {reps} passes in {dt:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
+        "steps": K, "warmup": args.warmup, "ms_per_step": ms_total / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": f"{w.name}: X {w.dtype} b={b} n={n}, dY b x m={m}, k={k}, per rank",
+                   "l2": "inputs exceed L2 (X %.0f MiB, dY %.0f MiB per step)" % (b * n * e / 2**20, b * m * e / 2**20)
+                   if b * n * e > 126 * 2**20 else "inputs fit L2: warm-cache numbers",
+                   "parallelism": f"replicas x{world}"},
+        "roofline": {"bound": "hbm", "kernel": "contract_main", "achieved": achieved, "peak": peak,
+                     "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": ab["contract"]},
+        "cpu_baseline": cpu,
+        "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": int(Xh.numel() * e + dYh.numel() * e), "d2h_bytes_per_step": int(dWh.numel() * 4),
+                "steps": Ke, "ms_per_step": ms_e2e / Ke, "checksum": checksum},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "stages": stages,
+        "memory_saved": saved,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--workload", default="c4", help="c1..c5; c4 (LLaMA-1B-shaped) is the headline configuration")
+    ap.add_argument("--k", type=int, default=0, help="override the workload's generator count")
+    ap.add_argument("--ref-tokens", type=int, default=16384, help="tokens per oracle pass (bounded sample)")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

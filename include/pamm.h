@@ -1,0 +1,202 @@
+/*
+ * pamm.h -- C ABI of the B200 (sm_100a) library for the hot path of
+ * Point-Approximate Matrix Multiplication (PAMM) on one fused Q|K|V layer.
+ *
+ * Notation follows the paper: A = X is the saved layer input (b tokens x n
+ * hidden), B = dY = [dQ|dK|dV] is the upstream gradient (b x m), C holds k
+ * generator rows of X, f in [0,k)^b assigns every row to a generator, alpha in
+ * R^b scales it, B~ (k x m) is the contracted gradient and dW~ = C^T B~ (n x m)
+ * approximates X^T dY.  epsilon = infinity throughout (the paper's chosen
+ * setting, Section 4.1): no row is dropped and beta = 1.
+ *
+ * Conventions for every entry point unless its comment says otherwise:
+ *  - Matrices are row-major with a leading dimension given in ELEMENTS.
+ *  - All matrix / vector pointers are DEVICE pointers owned by the caller.  The
+ *    library never allocates or frees device memory; scratch comes from the
+ *    caller as `workspace` (size from pamm_workspace_bytes).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *    only enqueue work; they never synchronise the host.
+ *  - Base pointers of X, dY, C, B~, dW must be 16-byte aligned and leading
+ *    dimensions must make every row start 16-byte aligned (ld * element size a
+ *    multiple of 16).  f, alpha, index arrays need 4-byte alignment, the
+ *    workspace 256-byte alignment.
+ *  - Argument errors (NULL, b < 1, k < 1, k > b, ld < columns, misalignment,
+ *    workspace too small, sizes over the documented limits) are reported
+ *    synchronously with nothing launched.  Unsupported dtype/shape
+ *    combinations return PAMM_ERR_UNSUPPORTED; there is no CPU fallback.
+ *  - Problems only the device can see (a generator index out of range, a
+ *    duplicated index, an assignment f_i outside [0,k), a bounded wait that ran
+ *    out) never trap: the kernel skips the access, ORs a bit into a per-device
+ *    status word and finishes.  Read it with pamm_last_device_status.
+ *  - Outputs are fully overwritten.  Results are deterministic: the same
+ *    inputs give bit-identical outputs from run to run.
+ */
+#ifndef PAMM_H_
+#define PAMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PAMM_OK = 0,
+    PAMM_ERR_INVALID_ARG = 1,
+    PAMM_ERR_UNSUPPORTED = 2,
+    PAMM_ERR_WORKSPACE = 3,
+    PAMM_ERR_CUDA = 4,
+    PAMM_ERR_TIMEOUT = 5,      /* a bounded device-side wait gave up            */
+    PAMM_ERR_BAD_INDEX = 6     /* device saw an out-of-range / duplicate index  */
+} pamm_status;
+
+typedef enum { PAMM_F32 = 0, PAMM_BF16 = 1 } pamm_dtype;
+
+/* Which scratch size is asked for. */
+typedef enum {
+    PAMM_WS_COMPRESS = 0,
+    PAMM_WS_CONTRACT = 1,            /* also covers pamm_contract_weight_grad */
+    PAMM_WS_STEP_HOST = 2            /* device arena of pamm_qkv_step_host    */
+} pamm_ws_kind;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* pamm_status_string(pamm_status s);
+
+/* Bytes of 256-byte-aligned device scratch the named call needs for these
+ * sizes (0 is a valid answer).  Returns (size_t)-1 for invalid sizes. */
+size_t pamm_workspace_bytes(pamm_ws_kind kind, int64_t b, int64_t n, int64_t m, int64_t k, pamm_dtype dt);
+
+/*
+ * Generator sampling on the host (Algorithm 1, "Sample indices I subset [b]
+ * uniformly without replacement, |I| = k").  The paper fixes no generator, so
+ * this library defines one: I = sort({pi_seed(0), ..., pi_seed(k-1)}) where
+ * pi_seed is a keyed pseudo-random permutation of [0,b) (a 6-round Feistel
+ * network on the smallest even-width power of two >= b, cycle-walked into
+ * range).  A pure function of (b, k, seed); the device path draws the same set.
+ * idx_out: HOST array of k int32, ascending.  No GPU is touched.
+ */
+pamm_status pamm_draw_indices_host(int64_t b, int64_t k, uint64_t seed, int32_t* idx_out);
+
+/*
+ * Step 1 -- choose generators (Algorithm 1: "Sample indices", "C <- A[I,:]",
+ * and the norms eta_C of the generator rows).
+ *   X        b x n, dtype dt, leading dimension ldx
+ *   idx_in   NULL: draw I from `seed` as pamm_draw_indices_host does (ascending);
+ *            else k caller-chosen row indices, used in the given order.  They
+ *            are checked on the device: an index outside [0,b) is clamped and a
+ *            repeated index is kept, both raising PAMM_ERR_BAD_INDEX in the
+ *            status word.
+ *   idx_out  k int32: the indices used
+ *   C        k x n, dtype dt, leading dimension ldc: exact copies of the rows
+ *   c_invnorm  2k fp32: [0,k) = 1/||C_j||, [k,2k) = 1/||C_j||^2; both 0 for a
+ *            zero row (such a generator scores 0 and yields alpha = 0)
+ * Limit: k <= 49152.
+ */
+pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
+                                   int64_t k, uint64_t seed, const int32_t* idx_in,
+                                   int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
+                                   void* stream);
+
+/*
+ * Step 2 -- compress (Section 3.2 "Compressing A", Eq. 1, Lemma 1; Algorithm 1
+ * lines "csim", "argmax", "alpha").  One streaming pass over X:
+ *   S = X C^T;  f_i = the lowest j maximising |S_ij| / ||C_j||  (equivalently
+ *   |csim(X_i, C_j)|, Lemma 1);  alpha_i = S_{i,f_i} / ||C_{f_i}||^2  (Eq. 1).
+ * Products are exact, sums are accumulated in fp32.  A zero row gets f = 0,
+ * alpha = 0.
+ *   f      b int32 (0-based)      alpha  b fp32
+ *   workspace  pamm_workspace_bytes(PAMM_WS_COMPRESS, ...) bytes
+ */
+pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
+                          const void* C, int64_t ldc, int64_t k, const float* c_invnorm,
+                          int32_t* f, float* alpha, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Steps 1+2 in one call (Algorithm 2, "C, alpha, f <- Compress(flatten(X), r)"):
+ * draws I from `seed` (or uses idx_in), then compresses.  Arguments as above.
+ */
+pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
+                                int64_t k, uint64_t seed, const int32_t* idx_in,
+                                int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
+                                int32_t* f, float* alpha, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Step 3 -- contract (Section 3.2 "Approximate Matrix Multiplication";
+ * Algorithm 1 ApproxMM: "B' <- alpha (.) B", "B~ <- index_add(B~, 0, f, B')"):
+ *   B~[j,:] = sum over {i : f_i = j} of alpha_i * dY[i,:]      (k x m, fp32)
+ * B' is never materialised.  dY is read once; rows are grouped by f with a
+ * stable counting sort, summed in fp32 in ascending row order inside fixed-size
+ * chunks, and chunk sums are added in ascending order -- no floating-point
+ * atomics, so the result is reproducible bit for bit.  A row whose f_i is
+ * outside [0,k) is skipped and raises PAMM_ERR_BAD_INDEX in the status word.
+ *   dY  b x m, dtype dt, leading dimension ldy     Btilde  k x m fp32, ldb
+ */
+pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy,
+                          int64_t b, int64_t m, pamm_dtype dt, int64_t k,
+                          float* Btilde, int64_t ldb, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Step 4 -- weight gradient (Algorithm 1 ApproxMM, "O~ <- C^T B~"; Algorithm 3,
+ * "grad W~ <- ApproxMM(C, alpha, f, grad Z)"):
+ *   dW[r,c] = sum_j C[j,r] * B~[j,c]                          (n x m, fp32)
+ *   C  k x n, dtype dt, ldc      Btilde  k x m fp32, ldb      dW  n x m fp32, ldw
+ */
+pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
+                             const float* Btilde, int64_t ldb, int64_t m,
+                             float* dW, int64_t ldw, void* stream);
+
+/*
+ * Steps 3+4 in one call (Algorithm 3, backward of the linear layer, the
+ * weight-gradient half): contract dY into B~ and multiply by C^T.  Btilde may
+ * be NULL, in which case B~ lives in the workspace only.
+ */
+pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n,
+                                      const int32_t* f, const float* alpha,
+                                      const void* dY, int64_t ldy, int64_t b, int64_t m, pamm_dtype dt,
+                                      int64_t k, float* Btilde, int64_t ldb,
+                                      float* dW, int64_t ldw,
+                                      void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * The whole path from HOST buffers (Algorithm 2's Compress followed by
+ * Algorithm 3's ApproxMM for one layer): copies X and dY host->device into the
+ * caller's device arena, runs steps 1-4 there, and copies dW (and, if the
+ * pointers are non-NULL, f and alpha) back to the host.  X_host / dY_host /
+ * dW_host should be pinned for the copies to be asynchronous.  `arena` is
+ * pamm_workspace_bytes(PAMM_WS_STEP_HOST, ...) bytes of device memory.
+ * The call enqueues everything on `stream` and returns; synchronise the stream
+ * before reading the host outputs.
+ */
+pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host,
+                               int64_t b, int64_t n, int64_t m, pamm_dtype dt,
+                               int64_t k, uint64_t seed,
+                               float* dW_host, int32_t* f_host, float* alpha_host,
+                               void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reads and clears the current device's status
+ * word.  Returns PAMM_OK, PAMM_ERR_TIMEOUT, PAMM_ERR_BAD_INDEX, or
+ * PAMM_ERR_CUDA if the stream itself reports an error.
+ */
+pamm_status pamm_last_device_status(void* stream);
+
+/*
+ * Measurement hooks (no counterpart in the paper).  pamm_launch_count returns
+ * the number of kernels this library has launched in this process.
+ * pamm_set_profile_events makes later calls record the two given cudaEvent_t
+ * (passed as void*, NULL to stop) on the call's stream immediately before and
+ * after the named step's main kernel, so a benchmark can time that kernel in
+ * place.  The events stay owned by the caller.  Not thread-safe.
+ */
+typedef enum { PAMM_PROF_COMPRESS = 0, PAMM_PROF_CONTRACT = 1, PAMM_PROF_WEIGHT_GRAD = 2 } pamm_prof_kind;
+unsigned long long pamm_launch_count(void);
+pamm_status pamm_set_profile_events(pamm_prof_kind kind, void* start_event, void* stop_event);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int pamm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PAMM_H_ */

@@ -1,0 +1,71 @@
+// Step 2 on CUDA cores: scoring S = X C^T, per-row argmax of |S_ij| / ||C_j||
+// (Lemma 1) and alpha (Eq. 1).  One warp streams one row of X with 16-byte
+// loads and keeps KC dot products per lane; a shuffle tree finishes each dot
+// product and every lane then holds the same totals, so the argmax needs no
+// further exchange.  This is the path for fp32 inputs and for small k, where
+// the contraction is too thin for tensor cores.
+#pragma once
+#include "pamm_common.cuh"
+
+namespace pamm {
+
+constexpr int CS_THREADS = 256;
+constexpr int CS_WARPS = CS_THREADS / 32;
+
+template <typename T, int KC>
+__global__ void __launch_bounds__(CS_THREADS)
+compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
+                     const T* __restrict__ C, int64_t ldc, int k,
+                     const float* __restrict__ c_invnorm,
+                     int32_t* __restrict__ f, float* __restrict__ alpha) {
+    constexpr int V = Vec16<T>::N;
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (int64_t)blockIdx.x * CS_WARPS + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * CS_WARPS;
+
+    for (int64_t i = warp0; i < b; i += nwarps) {
+        const T* xrow = X + i * ldx;
+        float best = -1.f, s_best = 0.f;
+        int j_best = 0;
+        for (int j0 = 0; j0 < k; j0 += KC) {
+            float acc[KC];
+#pragma unroll
+            for (int jj = 0; jj < KC; ++jj) acc[jj] = 0.f;
+            for (int64_t col = (int64_t)lane * V; col < n; col += 32 * V) {
+                float x[V];
+                load_vec<T>(xrow, col, n, x);
+#pragma unroll
+                for (int jj = 0; jj < KC; ++jj) {
+                    if (j0 + jj < k) {
+                        float c[V];
+                        load_vec<T>(C + (int64_t)(j0 + jj) * ldc, col, n, c);
+#pragma unroll
+                        for (int e = 0; e < V; ++e) acc[jj] = fmaf(x[e], c[e], acc[jj]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int jj = 0; jj < KC; ++jj) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) acc[jj] += __shfl_xor_sync(0xffffffffu, acc[jj], off);
+            }
+#pragma unroll
+            for (int jj = 0; jj < KC; ++jj) {
+                if (j0 + jj < k) {
+                    float score = fabsf(acc[jj]) * __ldg(c_invnorm + j0 + jj);
+                    if (score > best) {   // strict: the lowest index keeps a tie
+                        best = score;
+                        s_best = acc[jj];
+                        j_best = j0 + jj;
+                    }
+                }
+            }
+        }
+        if (lane == 0) {
+            f[i] = j_best;
+            alpha[i] = s_best * __ldg(c_invnorm + k + j_best);
+        }
+    }
+}
+
+}  // namespace pamm

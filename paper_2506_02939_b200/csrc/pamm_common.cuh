@@ -1,0 +1,122 @@
+// Shared device/host helpers of the PAMM sm_100a library: status word, storage
+// types, 16-byte vector access, the keyed permutation used for sampling.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/pamm.h"
+
+namespace pamm {
+
+// Bits ORed into the per-device status word by kernels (never a trap).
+enum : int { DEV_TIMEOUT = 1, DEV_BAD_INDEX = 2 };
+
+__device__ int g_status_word;
+
+__device__ __forceinline__ void raise_status(int bit) { atomicOr(&g_status_word, bit); }
+
+// ---- storage types ----------------------------------------------------------
+template <typename T> struct Vec16;   // 16 bytes of T
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    float v[4];
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    uint32_t w[4];
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Load up to 16 bytes of a row starting at element `col`; elements at or beyond
+// `ncols` read as zero.  `row` is 16-byte aligned and `col` a multiple of N.
+template <typename T>
+__device__ __forceinline__ void load_vec(const T* row, int64_t col, int64_t ncols, float (&out)[Vec16<T>::N]);
+
+template <>
+__device__ __forceinline__ void load_vec<float>(const float* row, int64_t col, int64_t ncols, float (&out)[4]) {
+    if (col + 4 <= ncols) {
+        float4 t = __ldg(reinterpret_cast<const float4*>(row + col));
+        out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) out[e] = (col + e < ncols) ? __ldg(row + col + e) : 0.f;
+    }
+}
+
+template <>
+__device__ __forceinline__ void load_vec<__nv_bfloat16>(const __nv_bfloat16* row, int64_t col, int64_t ncols,
+                                                        float (&out)[8]) {
+    if (col + 8 <= ncols) {
+        uint4 t = __ldg(reinterpret_cast<const uint4*>(row + col));
+        out[0] = bf16_lo(t.x); out[1] = bf16_hi(t.x); out[2] = bf16_lo(t.y); out[3] = bf16_hi(t.y);
+        out[4] = bf16_lo(t.z); out[5] = bf16_hi(t.z); out[6] = bf16_lo(t.w); out[7] = bf16_hi(t.w);
+    } else {
+        const unsigned short* r16 = reinterpret_cast<const unsigned short*>(row);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            out[e] = (col + e < ncols) ? __uint_as_float(((uint32_t)__ldg(r16 + col + e)) << 16) : 0.f;
+    }
+}
+
+// ---- keyed permutation of [0,b) used to sample generators ---------------------
+// A 6-round balanced Feistel network on w bits (w even, 2^w >= b), cycle-walked
+// until the value falls below b.  Round keys come from splitmix64(seed).
+struct PermKey {
+    uint32_t key[6];
+    uint32_t half_bits;
+    uint32_t half_mask;
+    uint32_t b;
+};
+
+__host__ __device__ inline uint64_t splitmix64(uint64_t x) {
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+
+__host__ __device__ inline PermKey make_perm_key(uint64_t seed, uint32_t b) {
+    PermKey pk;
+    uint32_t w = 2;
+    while (w < 32 && (1ull << w) < (uint64_t)b) w += 2;
+    pk.half_bits = w / 2;
+    pk.half_mask = (1u << (w / 2)) - 1u;
+    pk.b = b;
+    uint64_t s = seed;
+    for (int r = 0; r < 6; ++r) {
+        s = splitmix64(s);
+        pk.key[r] = (uint32_t)(s >> 32);
+    }
+    return pk;
+}
+
+__host__ __device__ inline uint32_t feistel_round_fn(uint32_t r, uint32_t key) {
+    uint32_t h = r * 0x9E3779B1u + key;
+    h ^= h >> 16; h *= 0x85EBCA6Bu;
+    h ^= h >> 13; h *= 0xC2B2AE35u;
+    h ^= h >> 16;
+    return h;
+}
+
+__host__ __device__ inline uint32_t perm_apply(const PermKey& pk, uint32_t x) {
+    // bounded cycle walk: the domain is < 4b, so the expected walk is < 4 steps
+    for (int walk = 0; walk < 4096; ++walk) {
+        uint32_t L = x >> pk.half_bits, R = x & pk.half_mask;
+        for (int r = 0; r < 6; ++r) {
+            uint32_t t = (L ^ feistel_round_fn(R, pk.key[r])) & pk.half_mask;
+            L = R;
+            R = t;
+        }
+        x = (L << pk.half_bits) | R;
+        if (x < pk.b) return x;
+    }
+    return x % pk.b;   // unreachable in practice; keeps the walk bounded
+}
+
+inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace pamm

@@ -1,0 +1,363 @@
+// C ABI of the PAMM sm_100a library: argument checks, kernel selection, launches.
+// Every step of the path runs in the kernels included below; nothing here
+// computes on the host apart from pamm_draw_indices_host.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "pamm_common.cuh"
+#include "select.cuh"
+#include "compress_simt.cuh"
+#include "compress_umma.cuh"
+#include "contract.cuh"
+#include "weight_grad_simt.cuh"
+#include "weight_grad_mma.cuh"
+
+using namespace pamm;
+
+namespace {
+
+inline size_t esize(pamm_dtype dt) { return dt == PAMM_BF16 ? 2 : 4; }
+inline bool dtype_ok(pamm_dtype dt) { return dt == PAMM_F32 || dt == PAMM_BF16; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline bool ld_ok(int64_t ld, int64_t cols, size_t es) { return ld >= cols && (ld * (int64_t)es) % 16 == 0; }
+inline pamm_status launch_status() { return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA; }
+constexpr int64_t MAX_ROWS = (1ll << 31) - 1024;   // row ids, counts and offsets are int32
+
+// Kernel launches issued so far (all streams), and optional event pairs that
+// bracket the dominant kernel of a step so a benchmark can time it in place.
+unsigned long long g_launches = 0;
+cudaEvent_t g_prof[3][2] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};
+inline void prof_begin(int kind, cudaStream_t st) { if (g_prof[kind][0]) cudaEventRecord(g_prof[kind][0], st); }
+inline void prof_end(int kind, cudaStream_t st) { if (g_prof[kind][1]) cudaEventRecord(g_prof[kind][1], st); }
+
+struct StepArena {
+    char *X, *dY, *C, *dW, *Bt, *ws;
+    float *invnorm, *alpha;
+    int32_t *idx, *f;
+    int64_t ldx, ldy, ldc, ldw, ldb;
+    size_t ws_bytes, bytes;
+};
+
+StepArena step_arena_layout(void* base, int64_t b, int64_t n, int64_t m, int64_t k, pamm_dtype dt) {
+    StepArena a;
+    const size_t es = esize(dt);
+    const int64_t v = 16 / (int64_t)es;
+    a.ldx = round_up(n, v); a.ldy = round_up(m, v); a.ldc = a.ldx;
+    a.ldw = round_up(m, 4); a.ldb = a.ldw;
+    char* p = (char*)base;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 256); return p ? p + o : (char*)0; };
+    a.X = take((size_t)b * a.ldx * es);
+    a.dY = take((size_t)b * a.ldy * es);
+    a.C = take((size_t)k * a.ldc * es);
+    a.invnorm = (float*)take((size_t)2 * k * 4);
+    a.idx = (int32_t*)take((size_t)k * 4);
+    a.f = (int32_t*)take((size_t)b * 4);
+    a.alpha = (float*)take((size_t)b * 4);
+    a.Bt = take((size_t)k * a.ldb * 4);
+    a.dW = take((size_t)n * a.ldw * 4);
+    a.ws_bytes = contract_ws_layout(nullptr, b, m, k).bytes;
+    a.ws = take(a.ws_bytes);
+    a.bytes = off;
+    return a;
+}
+
+template <typename T>
+pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int64_t k, uint64_t seed,
+                          const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
+                          cudaStream_t st) {
+    const size_t smem = (size_t)k * 4;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    const PermKey pk = make_perm_key(seed, (uint32_t)b);
+    const int grid = (int)((k + SEL_WARPS - 1) / SEL_WARPS);
+    select_kernel<T><<<grid, SEL_THREADS, smem, st>>>((const T*)X, ldx, b, n, (int)k, pk, idx_in, idx_out,
+                                                      (T*)C, ldc, c_invnorm);
+    g_launches += 1;
+    return launch_status();
+}
+
+template <typename T>
+pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
+                                 int64_t k, const float* c_invnorm, int32_t* f, float* alpha, cudaStream_t st) {
+    const int64_t want = (b + CS_WARPS - 1) / CS_WARPS;
+    const int grid = (int)std::min<int64_t>(want, 148 * 8);
+    prof_begin(PAMM_PROF_COMPRESS, st);
+    if (k <= 4)
+        compress_simt_kernel<T, 4><<<grid, CS_THREADS, 0, st>>>((const T*)X, ldx, b, n, (const T*)C, ldc, (int)k,
+                                                                c_invnorm, f, alpha);
+    else
+        compress_simt_kernel<T, 8><<<grid, CS_THREADS, 0, st>>>((const T*)X, ldx, b, n, (const T*)C, ldc, (int)k,
+                                                                c_invnorm, f, alpha);
+    prof_end(PAMM_PROF_COMPRESS, st);
+    g_launches += 1;
+    return launch_status();
+}
+
+template <typename T>
+pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
+                            int64_t k, float* Bt, int64_t ldb, const ContractWs& w, cudaStream_t st) {
+    constexpr int V = Vec16<T>::N;
+    const size_t hsmem = (size_t)k * 4;
+    if (hsmem > 48 * 1024 &&
+        cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    contract_hist_kernel<<<(int)w.nb, SORT_BLK, hsmem, st>>>(f, b, (int)k, w.hist);
+    contract_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(w.hist, (int)w.nb, (int)k, w.seg_start, w.chunk_base, w.chunk_seg);
+    contract_scatter_kernel<<<(int)w.nb, SORT_BLK, 0, st>>>(f, b, (int)k, w.hist, w.seg_start, w.perm);
+    const int64_t vecs = (m + V - 1) / V;
+    const int64_t slabs = (vecs + CT_MAX_THREADS - 1) / CT_MAX_THREADS;
+    const int threads = (int)round_up((vecs + slabs - 1) / slabs, 32);
+    dim3 grid((unsigned)w.max_chunks, (unsigned)slabs);
+    prof_begin(PAMM_PROF_CONTRACT, st);
+    contract_main_kernel<T><<<grid, threads, 0, st>>>(alpha, (const T*)dY, ldy, m, (int)k, w.seg_start, w.chunk_base,
+                                                      w.chunk_seg, w.perm, w.partials, w.m_pad);
+    prof_end(PAMM_PROF_CONTRACT, st);
+    g_launches += 5;
+    const int64_t items = k * (w.m_pad / 4);
+    contract_reduce_kernel<<<(int)((items + RED_THREADS - 1) / RED_THREADS), RED_THREADS, 0, st>>>(
+        w.partials, w.m_pad, m, (int)k, w.chunk_base, Bt, ldb);
+    return launch_status();
+}
+
+template <typename T>
+pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
+                                    int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
+    const int64_t items = n * ((m + 3) / 4);
+    prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
+    weight_grad_simt_kernel<T><<<(int)((items + WG_THREADS - 1) / WG_THREADS), WG_THREADS, 0, st>>>(
+        (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw);
+    prof_end(PAMM_PROF_WEIGHT_GRAD, st);
+    g_launches += 1;
+    return launch_status();
+}
+
+pamm_status check_select(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, int64_t k,
+                         int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!X || !idx_out || !C || !c_invnorm) return PAMM_ERR_INVALID_ARG;
+    if (b < 1 || n < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(ldx, n, esize(dt)) || !ld_ok(ldc, n, esize(dt))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(C, 16) || !aligned(idx_out, 4) || !aligned(c_invnorm, 4)) return PAMM_ERR_INVALID_ARG;
+    if (k > SEL_MAX_K) return PAMM_ERR_UNSUPPORTED;
+    return PAMM_OK;
+}
+
+pamm_status check_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C,
+                           int64_t ldc, int64_t k, const float* c_invnorm, int32_t* f, float* alpha) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!X || !C || !c_invnorm || !f || !alpha) return PAMM_ERR_INVALID_ARG;
+    if (b < 1 || n < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(ldx, n, esize(dt)) || !ld_ok(ldc, n, esize(dt))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(C, 16) || !aligned(f, 4) || !aligned(alpha, 4) || !aligned(c_invnorm, 4))
+        return PAMM_ERR_INVALID_ARG;
+    return PAMM_OK;
+}
+
+pamm_status check_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
+                           pamm_dtype dt, int64_t k, const float* Bt, int64_t ldb, bool bt_required,
+                           const void* ws, size_t ws_bytes) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!f || !alpha || !dY || (bt_required && !Bt)) return PAMM_ERR_INVALID_ARG;
+    if (b < 1 || m < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(ldy, m, esize(dt)) || (Bt && !ld_ok(ldb, m, 4))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(dY, 16) || (Bt && !aligned(Bt, 16)) || !aligned(f, 4) || !aligned(alpha, 4)) return PAMM_ERR_INVALID_ARG;
+    if (k > CT_MAX_K) return PAMM_ERR_UNSUPPORTED;
+    if (!ws || !aligned(ws, 256)) return PAMM_ERR_WORKSPACE;
+    if (ws_bytes < contract_ws_layout(nullptr, b, m, k).bytes) return PAMM_ERR_WORKSPACE;
+    return PAMM_OK;
+}
+
+pamm_status check_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
+                              int64_t ldb, int64_t m, float* dW, int64_t ldw) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!C || !Bt || !dW) return PAMM_ERR_INVALID_ARG;
+    if (k < 1 || n < 1 || m < 1) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(ldc, n, esize(dt)) || !ld_ok(ldb, m, 4) || !ld_ok(ldw, m, 4)) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(C, 16) || !aligned(Bt, 16) || !aligned(dW, 16)) return PAMM_ERR_INVALID_ARG;
+    return PAMM_OK;
+}
+
+pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
+                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, cudaStream_t st) {
+    if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+    if (compress_umma_supported(b, n, k))
+        return launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+    return launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+}
+
+pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
+                           int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
+    if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+    if (weight_grad_mma_supported(k, n, m))
+        return launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pamm_status_string(pamm_status s) {
+    switch (s) {
+        case PAMM_OK: return "ok";
+        case PAMM_ERR_INVALID_ARG: return "invalid argument";
+        case PAMM_ERR_UNSUPPORTED: return "unsupported dtype or shape";
+        case PAMM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case PAMM_ERR_CUDA: return "CUDA error";
+        case PAMM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case PAMM_ERR_BAD_INDEX: return "index out of range or duplicated on the device";
+    }
+    return "unknown status";
+}
+
+int pamm_version(void) { return 100; }
+
+unsigned long long pamm_launch_count(void) { return g_launches; }
+
+pamm_status pamm_set_profile_events(pamm_prof_kind kind, void* start_event, void* stop_event) {
+    if ((int)kind < 0 || (int)kind > 2) return PAMM_ERR_INVALID_ARG;
+    g_prof[kind][0] = (cudaEvent_t)start_event;
+    g_prof[kind][1] = (cudaEvent_t)stop_event;
+    return PAMM_OK;
+}
+
+size_t pamm_workspace_bytes(pamm_ws_kind kind, int64_t b, int64_t n, int64_t m, int64_t k, pamm_dtype dt) {
+    if (!dtype_ok(dt) || b < 1 || k < 1 || k > b || b > MAX_ROWS) return (size_t)-1;
+    switch (kind) {
+        case PAMM_WS_COMPRESS:
+            if (n < 1) return (size_t)-1;
+            return 0;
+        case PAMM_WS_CONTRACT:
+            if (m < 1) return (size_t)-1;
+            return contract_ws_layout(nullptr, b, m, k).bytes;
+        case PAMM_WS_STEP_HOST:
+            if (n < 1 || m < 1) return (size_t)-1;
+            return step_arena_layout(nullptr, b, n, m, k, dt).bytes;
+    }
+    return (size_t)-1;
+}
+
+pamm_status pamm_draw_indices_host(int64_t b, int64_t k, uint64_t seed, int32_t* idx_out) {
+    if (!idx_out || b < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    const PermKey pk = make_perm_key(seed, (uint32_t)b);
+    for (int64_t j = 0; j < k; ++j) idx_out[j] = (int32_t)perm_apply(pk, (uint32_t)j);
+    std::sort(idx_out, idx_out + k);
+    return PAMM_OK;
+}
+
+pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, int64_t k,
+                                   uint64_t seed, const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc,
+                                   float* c_invnorm, void* stream) {
+    pamm_status s = check_select(X, ldx, b, n, dt, k, idx_out, C, ldc, c_invnorm);
+    if (s != PAMM_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    return dt == PAMM_F32 ? launch_select<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st)
+                          : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
+}
+
+pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
+                          int64_t k, const float* c_invnorm, int32_t* f, float* alpha, void* workspace,
+                          size_t ws_bytes, void* stream) {
+    (void)workspace; (void)ws_bytes;
+    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+    if (s != PAMM_OK) return s;
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, (cudaStream_t)stream);
+}
+
+pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, int64_t k,
+                                uint64_t seed, const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc,
+                                float* c_invnorm, int32_t* f, float* alpha, void* workspace, size_t ws_bytes,
+                                void* stream) {
+    (void)workspace; (void)ws_bytes;
+    pamm_status s = check_select(X, ldx, b, n, dt, k, idx_out, C, ldc, c_invnorm);
+    if (s != PAMM_OK) return s;
+    s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+    if (s != PAMM_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = dt == PAMM_F32 ? launch_select<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st)
+                       : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
+    if (s != PAMM_OK) return s;
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, st);
+}
+
+pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
+                          pamm_dtype dt, int64_t k, float* Btilde, int64_t ldb, void* workspace, size_t ws_bytes,
+                          void* stream) {
+    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, workspace, ws_bytes);
+    if (s != PAMM_OK) return s;
+    const ContractWs w = contract_ws_layout(workspace, b, m, k);
+    cudaStream_t st = (cudaStream_t)stream;
+    return dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st)
+                          : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st);
+}
+
+pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Btilde,
+                             int64_t ldb, int64_t m, float* dW, int64_t ldw, void* stream) {
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+    if (s != PAMM_OK) return s;
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream);
+}
+
+pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, const int32_t* f, const float* alpha,
+                                      const void* dY, int64_t ldy, int64_t b, int64_t m, pamm_dtype dt, int64_t k,
+                                      float* Btilde, int64_t ldb, float* dW, int64_t ldw, void* workspace,
+                                      size_t ws_bytes, void* stream) {
+    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, false, workspace, ws_bytes);
+    if (s != PAMM_OK) return s;
+    const ContractWs w = contract_ws_layout(workspace, b, m, k);
+    float* Bt = Btilde ? Btilde : w.btilde;
+    const int64_t ldbt = Btilde ? ldb : w.m_pad;
+    s = check_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dW, ldw);
+    if (s != PAMM_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    s = dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Bt, ldbt, w, st)
+                       : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Bt, ldbt, w, st);
+    if (s != PAMM_OK) return s;
+    return do_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dW, ldw, st);
+}
+
+pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host, int64_t b, int64_t n, int64_t m,
+                               pamm_dtype dt, int64_t k, uint64_t seed, float* dW_host, int32_t* f_host,
+                               float* alpha_host, void* arena, size_t arena_bytes, void* stream) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!X_host || !dY_host || !dW_host) return PAMM_ERR_INVALID_ARG;
+    if (b < 1 || n < 1 || m < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (k > SEL_MAX_K) return PAMM_ERR_UNSUPPORTED;
+    if (!arena || !aligned(arena, 256)) return PAMM_ERR_WORKSPACE;
+    const StepArena a = step_arena_layout(arena, b, n, m, k, dt);
+    if (arena_bytes < a.bytes) return PAMM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = esize(dt);
+    if (cudaMemcpy2DAsync(a.X, a.ldx * es, X_host, n * es, n * es, b, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpy2DAsync(a.dY, a.ldy * es, dY_host, m * es, m * es, b, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    pamm_status s = pamm_compress_fused(a.X, a.ldx, b, n, dt, k, seed, nullptr, a.idx, a.C, a.ldc, a.invnorm, a.f,
+                                        a.alpha, nullptr, 0, stream);
+    if (s != PAMM_OK) return s;
+    s = pamm_contract_weight_grad(a.C, a.ldc, n, a.f, a.alpha, a.dY, a.ldy, b, m, dt, k, (float*)a.Bt, a.ldb,
+                                  (float*)a.dW, a.ldw, a.ws, a.ws_bytes, stream);
+    if (s != PAMM_OK) return s;
+    if (cudaMemcpy2DAsync(dW_host, m * 4, a.dW, a.ldw * 4, m * 4, n, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    if (f_host && cudaMemcpyAsync(f_host, a.f, (size_t)b * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    if (alpha_host && cudaMemcpyAsync(alpha_host, a.alpha, (size_t)b * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    return PAMM_OK;
+}
+
+pamm_status pamm_last_device_status(void* stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PAMM_ERR_CUDA;
+    int word = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int)) != cudaSuccess) return PAMM_ERR_CUDA;
+    if (word && cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return PAMM_ERR_CUDA;
+    if (word & DEV_TIMEOUT) return PAMM_ERR_TIMEOUT;
+    if (word & DEV_BAD_INDEX) return PAMM_ERR_BAD_INDEX;
+    return PAMM_OK;
+}
+
+}  // extern "C"

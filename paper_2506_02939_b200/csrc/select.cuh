@@ -1,0 +1,78 @@
+// Step 1: generator selection (Algorithm 1: "Sample indices I", "C <- A[I,:]",
+// and the norms of the generator rows).  One launch, no cross-CTA dependency:
+// every CTA recomputes the k candidate indices in shared memory, then each of
+// its warps ranks one candidate (rank = sorted position), copies that row of X
+// into C and accumulates its squared norm in fp64.
+#pragma once
+#include "pamm_common.cuh"
+
+namespace pamm {
+
+constexpr int SEL_THREADS = 256;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int64_t SEL_MAX_K = 49152;   // k * 4 bytes of dynamic shared memory
+
+template <typename T>
+__global__ void __launch_bounds__(SEL_THREADS)
+select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k, PermKey pk,
+              const int32_t* __restrict__ idx_in, int32_t* __restrict__ idx_out,
+              T* __restrict__ C, int64_t ldc, float* __restrict__ c_invnorm) {
+    extern __shared__ int32_t s_vals[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int j = tid; j < k; j += SEL_THREADS)
+        s_vals[j] = idx_in ? idx_in[j] : (int32_t)perm_apply(pk, (uint32_t)j);
+    __syncthreads();
+
+    const int j = blockIdx.x * SEL_WARPS + warp;
+    if (j >= k) return;
+    int32_t val = s_vals[j];
+
+    // rank among all candidates, and a duplicate count (warp-wide)
+    int smaller = 0, dup = 0;
+    for (int t = lane; t < k; t += 32) {
+        int32_t o = s_vals[t];
+        smaller += (o < val);
+        dup += (o == val && t != j);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        smaller += __shfl_xor_sync(0xffffffffu, smaller, off);
+        dup += __shfl_xor_sync(0xffffffffu, dup, off);
+    }
+    int slot;
+    if (idx_in) {
+        slot = j;   // caller's order
+        bool bad = dup > 0;
+        if (val < 0) { val = 0; bad = true; }
+        if ((int64_t)val >= b) { val = (int32_t)(b - 1); bad = true; }
+        if (bad && lane == 0) raise_status(DEV_BAD_INDEX);
+    } else {
+        slot = smaller;   // distinct by construction: rank = ascending position
+    }
+
+    constexpr int V = Vec16<T>::N;
+    const T* src = X + (int64_t)val * ldx;
+    T* dst = C + (int64_t)slot * ldc;
+    double q = 0.0;
+    for (int64_t col = (int64_t)lane * V; col < n; col += 32 * V) {
+        float x[V];
+        load_vec<T>(src, col, n, x);
+        if (col + V <= n) {
+            *reinterpret_cast<uint4*>(dst + col) = __ldg(reinterpret_cast<const uint4*>(src + col));
+        } else {
+            for (int e = 0; e < V && col + e < n; ++e) dst[col + e] = src[col + e];
+        }
+#pragma unroll
+        for (int e = 0; e < V; ++e) q += (double)x[e] * (double)x[e];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) q += __shfl_xor_sync(0xffffffffu, q, off);
+    if (lane == 0) {
+        idx_out[slot] = val;
+        c_invnorm[slot] = (q > 0.0) ? (float)(1.0 / sqrt(q)) : 0.f;
+        c_invnorm[k + slot] = (q > 0.0) ? (float)(1.0 / q) : 0.f;
+    }
+}
+
+}  // namespace pamm

@@ -1,0 +1,213 @@
+"""Thin binding to the PAMM CUDA library (C ABI declared in ``include/pamm.h``).
+
+Argument marshalling only: every step of the path runs in the library's kernels.
+torch is used for device memory and streams.  Importing this module fails
+loudly when the library has not been built; there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libpamm_b200.so"
+if not _LIB_PATH.exists():
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2506_02939_b200.build` "
+        "(nvcc, sm_100a). The PAMM path has no fallback.")
+_lib = ctypes.CDLL(str(_LIB_PATH))
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_INDEX = range(7)
+F32, BF16 = 0, 1
+WS_COMPRESS, WS_CONTRACT, WS_STEP_HOST = 0, 1, 2
+
+_i64, _vp, _ci, _u64, _sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_uint64, ctypes.c_size_t
+
+_SIGNATURES = {
+    "pamm_status_string": ([_ci], ctypes.c_char_p),
+    "pamm_version": ([], _ci),
+    "pamm_workspace_bytes": ([_ci, _i64, _i64, _i64, _i64, _ci], _sz),
+    "pamm_draw_indices_host": ([_i64, _i64, _u64, _vp], _ci),
+    "pamm_select_generators": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp], _ci),
+    "pamm_compress": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_compress_fused": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_contract": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
+    "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
+    "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
+    "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_last_device_status": ([_vp], _ci),
+    "pamm_launch_count": ([], ctypes.c_ulonglong),
+    "pamm_set_profile_events": ([_ci, _vp, _vp], _ci),
+}
+for _name, (_args, _res) in _SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.argtypes, _fn.restype = _args, _res
+
+EXPORTED = tuple(_SIGNATURES)
+
+
+class PammError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+def status_string(code: int) -> str:
+    return _lib.pamm_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(_lib.pamm_version())
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise PammError(code, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"PAMM inputs are float32 or bfloat16, got {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _ld(t: torch.Tensor) -> int:
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("need a 2-D row-major tensor (a row stride is allowed)")
+    return t.stride(0)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def workspace_bytes(kind: int, b: int, n: int, m: int, k: int, dtype: int) -> int:
+    r = _lib.pamm_workspace_bytes(kind, b, n, m, k, dtype)
+    if r == ctypes.c_size_t(-1).value:
+        raise PammError(ERR_INVALID_ARG, "pamm_workspace_bytes")
+    return int(r)
+
+
+def alloc_workspace(kind: int, b: int, n: int, m: int, k: int, dtype: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(256, workspace_bytes(kind, b, n, m, k, dtype)), dtype=torch.uint8, device=device)
+
+
+def draw_indices_host(b: int, k: int, seed: int) -> torch.Tensor:
+    out = torch.empty(k, dtype=torch.int32)
+    _check(_lib.pamm_draw_indices_host(b, k, seed, _ptr(out)), "pamm_draw_indices_host")
+    return out
+
+
+def select_generators(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, stream=None):
+    b, n = X.shape
+    idx_out = torch.empty(k, dtype=torch.int32, device=X.device) if idx_out is None else idx_out
+    C = torch.empty((k, n), dtype=X.dtype, device=X.device) if C is None else C
+    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=X.device) if c_invnorm is None else c_invnorm
+    _check(_lib.pamm_select_generators(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out),
+                                       _ptr(C), _ld(C), _ptr(c_invnorm), _stream(stream)), "pamm_select_generators")
+    return idx_out, C, c_invnorm
+
+
+def compress(X, C, c_invnorm, f=None, alpha=None, workspace=None, stream=None):
+    b, n = X.shape
+    k = C.shape[0]
+    f = torch.empty(b, dtype=torch.int32, device=X.device) if f is None else f
+    alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
+    ws_bytes = 0 if workspace is None else workspace.numel()
+    _check(_lib.pamm_compress(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), _ptr(f),
+                              _ptr(alpha), _ptr(workspace), ws_bytes, _stream(stream)), "pamm_compress")
+    return f, alpha
+
+
+def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, f=None, alpha=None,
+                   workspace=None, stream=None):
+    b, n = X.shape
+    dev = X.device
+    idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
+    C = torch.empty((k, n), dtype=X.dtype, device=dev) if C is None else C
+    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
+    f = torch.empty(b, dtype=torch.int32, device=dev) if f is None else f
+    alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
+    ws_bytes = 0 if workspace is None else workspace.numel()
+    _check(_lib.pamm_compress_fused(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out), _ptr(C),
+                                    _ld(C), _ptr(c_invnorm), _ptr(f), _ptr(alpha), _ptr(workspace), ws_bytes,
+                                    _stream(stream)), "pamm_compress_fused")
+    return idx_out, C, c_invnorm, f, alpha
+
+
+def contract(f, alpha, dY, k: int, Btilde=None, workspace=None, stream=None):
+    b, m = dY.shape
+    Btilde = torch.empty((k, m), dtype=torch.float32, device=dY.device) if Btilde is None else Btilde
+    if workspace is None:
+        workspace = alloc_workspace(WS_CONTRACT, b, 1, m, k, _dt(dY), dY.device)
+    _check(_lib.pamm_contract(_ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde), _ld(Btilde),
+                              _ptr(workspace), workspace.numel(), _stream(stream)), "pamm_contract")
+    return Btilde
+
+
+def weight_grad(C, Btilde, dW=None, stream=None):
+    k, n = C.shape
+    m = Btilde.shape[1]
+    dW = torch.empty((n, m), dtype=torch.float32, device=C.device) if dW is None else dW
+    _check(_lib.pamm_weight_grad(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW),
+                                 _stream(stream)), "pamm_weight_grad")
+    return dW
+
+
+def contract_weight_grad(C, f, alpha, dY, Btilde=None, dW=None, workspace=None, stream=None):
+    k, n = C.shape
+    b, m = dY.shape
+    dW = torch.empty((n, m), dtype=torch.float32, device=C.device) if dW is None else dW
+    if workspace is None:
+        workspace = alloc_workspace(WS_CONTRACT, b, n, m, k, _dt(dY), dY.device)
+    _check(_lib.pamm_contract_weight_grad(_ptr(C), _ld(C), n, _ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY),
+                                          k, _ptr(Btilde), 0 if Btilde is None else _ld(Btilde), _ptr(dW), _ld(dW),
+                                          _ptr(workspace), workspace.numel(), _stream(stream)),
+           "pamm_contract_weight_grad")
+    return dW
+
+
+def qkv_step_host(X_host, dY_host, k: int, seed: int, dW_host, arena, f_host=None, alpha_host=None, stream=None):
+    """Whole path from (pinned) host tensors; ``arena`` is device scratch."""
+    b, n = X_host.shape
+    m = dY_host.shape[1]
+    if not (X_host.is_contiguous() and dY_host.is_contiguous() and dW_host.is_contiguous()):
+        raise ValueError("host tensors must be contiguous")
+    _check(_lib.pamm_qkv_step_host(_ptr(X_host), _ptr(dY_host), b, n, m, _dt(X_host), k, seed, _ptr(dW_host),
+                                   _ptr(f_host), _ptr(alpha_host), _ptr(arena), arena.numel(), _stream(stream)),
+           "pamm_qkv_step_host")
+    return dW_host
+
+
+def last_device_status(stream=None) -> int:
+    return int(_lib.pamm_last_device_status(_stream(stream)))
+
+
+PROF_COMPRESS, PROF_CONTRACT, PROF_WEIGHT_GRAD = 0, 1, 2
+
+
+def launch_count() -> int:
+    return int(_lib.pamm_launch_count())
+
+
+def set_profile_events(kind: int, start=None, stop=None) -> None:
+    """Record torch CUDA events (already recorded once, so their handles exist) around a step's main kernel."""
+    a = None if start is None else ctypes.c_void_p(start.cuda_event)
+    b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+    _check(_lib.pamm_set_profile_events(kind, a, b), "pamm_set_profile_events")
+
+
+def saved_bytes(b: int, n: int, k: int, dtype: int) -> dict:
+    """Bytes kept for the backward pass: X itself versus (C, f int32, alpha fp32)."""
+    e = 2 if dtype == BF16 else 4
+    full = b * n * e
+    kept = k * n * e + 8 * b
+    return dict(full=full, pamm=kept, ratio=full / kept, scalars_full=b * n, scalars_pamm=k * n + 2 * b)

@@ -1,0 +1,218 @@
+"""Parity of the CUDA path (called through the C ABI) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pamm_oracle as orc
+from paper_2506_02939_b200 import build as pamm_build, synth
+
+pamm_build.build()
+from paper_2506_02939_b200 import pamm  # noqa: E402
+from tests import parity  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+def _idx(b, k, seed):
+    return np.sort(np.random.default_rng(seed).choice(b, size=k, replace=False)).astype(np.int32)
+
+
+# (b, n, m, k, dtype): several tiles, ragged tails in every dimension, k = 1
+SMALL = [
+    (300, 72, 40, 5, "f32"),
+    (1000, 136, 264, 17, "bf16"),
+    (4133, 512, 520, 64, "bf16"),
+    (777, 2056, 1032, 128, "bf16"),
+    (2500, 200, 96, 1, "bf16"),
+    (1027, 516, 772, 4, "f32"),
+    (640, 64, 6152, 96, "bf16"),
+    (129, 8, 8, 129, "bf16"),
+    (5000, 1024, 256, 256, "bf16"),
+]
+
+
+@pytest.mark.parametrize("b,n,m,k,dtype", SMALL)
+@pytest.mark.parametrize("fused", [True, False])
+def test_small_cases(b, n, m, k, dtype, fused):
+    X, dY = synth.random_case(b, n, m, dtype, seed=b + k, centres=max(2, k // 2), dy_scale=1e-3)
+    rep = parity.run_and_compare(X, dY, k, seed=7 + k, fused=fused)
+    assert rep.unexplained == 0
+
+
+def test_ragged_columns_with_padded_leading_dimension():
+    # n and m are not multiples of the 16-byte vector; the row stride is
+    X, dY = synth.random_case(700, 70, 45, "f32", seed=3, centres=6)
+    parity.run_and_compare(X, dY, 9, seed=1, ldx=72, ldy=48)
+    X, dY = synth.random_case(700, 67, 83, "bf16", seed=4, centres=6)
+    parity.run_and_compare(X, dY, 9, seed=1, ldx=72, ldy=88)
+
+
+def test_k_equals_b_reproduces_exact_product():
+    X, dY = synth.random_case(384, 96, 80, "bf16", seed=5)
+    rep = parity.run_and_compare(X, dY, 384, idx_in=np.arange(384, dtype=np.int32))
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, 384, 0, idx_in=torch.arange(384, dtype=torch.int32, device="cuda"))
+    assert torch.equal(f.cpu(), torch.arange(384, dtype=torch.int32))
+    assert torch.allclose(alpha, torch.ones_like(alpha), rtol=1e-6, atol=0)
+    dW = pamm.contract_weight_grad(C, f, alpha, dYd).cpu().numpy()
+    exact = synth.to_f64(X).T @ synth.to_f64(dY)
+    assert parity.rel_fro(dW, exact) <= 1e-2
+    assert parity.rel_fro(dW, exact) <= 1e-4      # in fact only fp32 rounding remains
+
+
+def test_rank_one_input_reproduces_exact_product():
+    rng = np.random.default_rng(6)
+    u = (rng.integers(1, 9, size=512) * rng.choice([-1, 1], size=512)).astype(np.float32)
+    v = rng.integers(-8, 9, size=64).astype(np.float32)
+    v[0] = 5
+    X = np.outer(u, v).astype(np.float32)
+    _, dY = synth.random_case(512, 64, 48, "f32", seed=7)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, 3, 11)
+    dW = pamm.contract_weight_grad(C, f, alpha, dYd).cpu().numpy()
+    exact = X.astype(np.float64).T @ dY.astype(np.float64)
+    assert parity.rel_fro(dW, exact) <= 1e-5
+    # every generator ties on every row: whatever f the GPU picked, the oracle calls it a near-tie
+    rep = parity.run_and_compare(X, dY, 3, seed=11)
+    assert rep.unexplained == 0 and rep.explained_by_rounding == 0
+
+
+def test_padding_rows_share_f_and_alpha_and_zero_rows():
+    inp = synth.make_inputs("c2", num_seqs=16)
+    X, dY = inp.X, inp.dY
+    k = 8
+    parity.run_and_compare(X, dY, k, seed=3)
+    # force a zero generator and a duplicated generator row through caller-chosen indices
+    pads = inp.pad_rows
+    zero_rows = pads[np.all((X[pads] & 0x7FFF) == 0, axis=1)]
+    dup_rows = pads[~np.all((X[pads] & 0x7FFF) == 0, axis=1)]
+    assert len(zero_rows) > 2 and len(dup_rows) > 2
+    idx = np.array([5, dup_rows[0], 900, zero_rows[0], dup_rows[1], 2000], np.int32)
+    rep = parity.run_and_compare(X, dY, len(idx), idx_in=idx)
+    Xd = parity.to_device(X)
+    _, C, invn, f, alpha = pamm.compress_fused(Xd, len(idx), 0, idx_in=torch.from_numpy(idx).cuda())
+    f, alpha = f.cpu().numpy(), alpha.cpu().numpy()
+    assert np.all(f[dup_rows] == 1) and np.all(alpha[dup_rows] == alpha[dup_rows[0]])   # lowest of the twins
+    assert abs(alpha[dup_rows[0]] - 1.0) < 1e-6
+    assert np.all(f[zero_rows] == 0) and np.all(alpha[zero_rows] == 0.0)
+    assert not np.any(f == 3) and np.all(np.isfinite(alpha))
+
+
+def test_results_are_bit_reproducible():
+    X, dY = synth.random_case(3000, 256, 520, "bf16", seed=8, centres=20)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    outs = []
+    for _ in range(3):
+        idx, C, invn, f, alpha = pamm.compress_fused(Xd, 48, 5)
+        Bt = torch.empty((48, 520), dtype=torch.float32, device="cuda")
+        dW = pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt)
+        outs.append([t.clone() for t in (idx, C, invn, f, alpha, Bt, dW)])
+    for o in outs[1:]:
+        for a, b_ in zip(outs[0], o):
+            assert torch.equal(a.view(torch.uint8) if a.dtype == torch.bfloat16 else a,
+                               b_.view(torch.uint8) if b_.dtype == torch.bfloat16 else b_)
+
+
+def test_outputs_stay_inside_their_buffers():
+    b, n, m, k = 1500, 136, 264, 24
+    X, dY = synth.random_case(b, n, m, "bf16", seed=9, centres=10)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    G = 64
+
+    def guarded(shape, dtype):
+        numel = int(np.prod(shape))
+        raw = torch.full((numel + 2 * G,), -7, dtype=dtype, device="cuda") if dtype != torch.bfloat16 else \
+            torch.full((numel + 2 * G,), -7.0, dtype=dtype, device="cuda")
+        return raw, raw[G:G + numel].view(shape)
+
+    raws = {}
+    raws["idx"], idx = guarded((k,), torch.int32)
+    raws["C"], C = guarded((k, n), torch.bfloat16)
+    raws["invn"], invn = guarded((2 * k,), torch.float32)
+    raws["f"], f = guarded((b,), torch.int32)
+    raws["alpha"], alpha = guarded((b,), torch.float32)
+    raws["Bt"], Bt = guarded((k, m), torch.float32)
+    raws["dW"], dW = guarded((n, m), torch.float32)
+    need = pamm.workspace_bytes(pamm.WS_CONTRACT, b, n, m, k, pamm.BF16)
+    ws_raw = torch.full((need + 512,), 0x5A, dtype=torch.uint8, device="cuda")
+    ws = ws_raw[256:256 + need]
+    pamm.compress_fused(Xd, k, 2, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha)
+    pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt, dW=dW, workspace=ws)
+    assert pamm.last_device_status() == pamm.OK
+    for name, raw in raws.items():
+        head, tail = raw[:G].float().cpu(), raw[-G:].float().cpu()
+        assert torch.all(head == -7) and torch.all(tail == -7), name
+    assert torch.all(ws_raw[:256] == 0x5A) and torch.all(ws_raw[-256:] == 0x5A)
+    assert torch.all(torch.isfinite(dW))
+
+
+def test_device_side_problems_raise_a_status_not_a_fault():
+    X, dY = synth.random_case(256, 64, 32, "f32", seed=10)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    assert pamm.last_device_status() == pamm.OK
+    bad = torch.tensor([3, 999, 7, 7], dtype=torch.int32, device="cuda")     # out of range + duplicate
+    idx, C, invn = pamm.select_generators(Xd, 4, idx_in=bad)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
+    assert pamm.last_device_status() == pamm.OK                               # reading clears it
+    assert idx.cpu().tolist() == [3, 255, 7, 7]
+    f = torch.zeros(256, dtype=torch.int32, device="cuda")
+    f[10] = 4
+    f[11] = -1
+    alpha = torch.ones(256, dtype=torch.float32, device="cuda")
+    Bt = pamm.contract(f, alpha, dYd, 4)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
+    keep = np.ones(256, bool)
+    keep[[10, 11]] = False
+    assert np.allclose(Bt[0].cpu().numpy(), dY[keep].astype(np.float64).sum(axis=0), rtol=1e-4, atol=1e-6)
+    assert torch.all(Bt[1:] == 0)
+
+
+def test_unfused_stage_inputs_from_elsewhere():
+    # contract / weight_grad accept any (f, alpha, B~), not only what compress produced
+    rng = np.random.default_rng(12)
+    b, m, k, n = 2000, 300, 10, 40
+    _, dY = synth.random_case(b, 8, m, "bf16", seed=13)
+    f = rng.integers(0, k, size=b).astype(np.int32)
+    f[f == 4] = 5                                                     # an empty segment
+    a = rng.standard_normal(b).astype(np.float32)
+    Bt = pamm.contract(torch.from_numpy(f).cuda(), torch.from_numpy(a).cuda(), parity.to_device(dY), k)
+    ref = orc.contract(f, a.astype(np.float64), dY, k)
+    assert parity.rel_fro(Bt.cpu().numpy(), ref) <= 1e-5
+    assert torch.all(Bt[4] == 0)
+    Cb, _ = synth.random_case(k, n, 8, "bf16", seed=14)
+    dW = pamm.weight_grad(parity.to_device(Cb), Bt)
+    ref = orc.weight_grad(synth.to_f64(Cb), Bt.cpu().numpy().astype(np.float64))
+    assert parity.rel_fro(dW.cpu().numpy(), ref) <= 1e-4
+
+
+def test_host_buffer_step_matches_device_path():
+    X, dY = synth.random_case(1200, 128, 200, "bf16", seed=15, centres=12, dy_scale=1e-3)
+    Xh = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).pin_memory()
+    dYh = torch.from_numpy(dY.view(np.int16)).view(torch.bfloat16).pin_memory()
+    dWh = torch.empty((128, 200), dtype=torch.float32).pin_memory()
+    fh = torch.empty(1200, dtype=torch.int32).pin_memory()
+    ah = torch.empty(1200, dtype=torch.float32).pin_memory()
+    arena = pamm.alloc_workspace(pamm.WS_STEP_HOST, 1200, 128, 200, 16, pamm.BF16)
+    pamm.qkv_step_host(Xh, dYh, 16, 21, dWh, arena, f_host=fh, alpha_host=ah)
+    assert pamm.last_device_status() == pamm.OK
+    idx, C, invn, f, alpha = pamm.compress_fused(Xh.cuda(), 16, 21)
+    dW = pamm.contract_weight_grad(C, f, alpha, dYh.cuda())
+    assert torch.equal(fh, f.cpu()) and torch.equal(ah, alpha.cpu()) and torch.equal(dWh, dW.cpu())
+
+
+# ---- the five workloads at full size, in the launch configuration the benchmark times ----
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c4", "c5"])
+def test_workload_full_size(name):
+    inp = synth.make_inputs(name)
+    w = inp.workload
+    rep = parity.run_and_compare(inp.X, inp.dY, w.ks[0], seed=w.index_seed)
+    print(name, rep.err, "mismatch", rep.mismatches, "near-tie", rep.near_tie, "rounding", rep.explained_by_rounding)
+
+
+def test_workload_c3_ratio_sweep():
+    inp = synth.make_inputs("c3")
+    w = inp.workload
+    for k in w.ks:
+        rep = parity.run_and_compare(inp.X, inp.dY, k, seed=w.index_seed)
+        print("c3", k, rep.err, "mismatch", rep.mismatches, "near-tie", rep.near_tie, "rounding", rep.explained_by_rounding)
