@@ -1,7 +1,261 @@
+// Step 2 on tensor cores (bf16 inputs): S = X C^T with tcgen05.mma into tensor
+// memory, then per-row argmax of |S_ij| / ||C_j|| (Lemma 1) and alpha (Eq. 1).
+//
+// One streaming pass over X.  The rows are cut into equal contiguous ranges, one
+// per CTA (one CTA per SM, a single balanced wave).  Inside a CTA:
+//   warp 0     TMA producer: X tiles (32-row boxes, so a ragged last tile costs
+//              only the bytes it needs) and the matching C tile, 64 columns of
+//              the hidden dimension per pipeline stage, 128-byte swizzle
+//   warp 1     issues tcgen05.mma (M = 128 rows, N = generators of the chunk,
+//              K = 16 per instruction), fp32 accumulators in TMEM, two buffers
+//   warps 2-5  epilogue: each thread owns one row (TMEM lane), reads its scores
+//              with tcgen05.ld and scans them in ascending j with a strict '>'
+//              so the lowest index wins ties; the epilogue of one tile overlaps
+//              the MMAs of the next
+// C is small (k x n) and is re-read per row tile from L2; with MT = 2 two row
+// tiles share every C tile.  For k > 256 the generators are processed in chunks
+// with a running (best score, argmax, dot product) per row.
 #pragma once
 #include "pamm_common.cuh"
+#include "sm100_ptx.cuh"
+
 namespace pamm {
-inline bool compress_umma_supported(int64_t, int64_t, int64_t) { return false; }
-inline pamm_status launch_compress_umma(const void*, int64_t, int64_t, int64_t, const void*, int64_t, int64_t,
-                                        const float*, int32_t*, float*, cudaStream_t) { return PAMM_ERR_UNSUPPORTED; }
+
+constexpr int CU_THREADS = 192;
+constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
+constexpr int CU_TILE_M = 128;
+constexpr int CU_BOX_ROWS = 32;
+constexpr int CU_X_TILE_BYTES = CU_TILE_M * 128;   // 16 KiB
+constexpr int CU_MAX_K = 4096;                 // 1/||C_j|| and 1/||C_j||^2 live in shared memory
+constexpr int CU_SMEM_BUDGET = 200 * 1024;
+
+struct CompressUmmaPlan {
+    int mt;            // row tiles (of 128) per super tile: 2 when the chunk has <= 128 generators
+    int n_chunk;       // generators per chunk, padded to a multiple of 16 (<= 256)
+    int num_chunks;
+    int stages;
+    int stage_bytes;
+    int tmem_cols;
+    int rows_per_cta;
+    int grid;
+    size_t smem_bytes;
+};
+
+inline bool compress_umma_supported(int64_t b, int64_t n, int64_t k) {
+    return k >= 16 && k <= CU_MAX_K && n >= 8 && b >= 1 && n < (1ll << 31);
 }
+
+inline CompressUmmaPlan compress_umma_plan(int64_t b, int64_t k, int sms) {
+    CompressUmmaPlan p;
+    const int npad = (int)round_up(k, 16);
+    p.num_chunks = (npad + 255) / 256;
+    p.n_chunk = (int)round_up((npad + p.num_chunks - 1) / p.num_chunks, 16);
+    p.mt = p.n_chunk <= 128 ? 2 : 1;
+    p.stage_bytes = p.mt * CU_X_TILE_BYTES + p.n_chunk * 128;
+    p.stages = std::min(8, CU_SMEM_BUDGET / p.stage_bytes);
+    int cols = 2 * p.mt * p.n_chunk;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < cols) p.tmem_cols *= 2;
+    const int64_t per = (b + sms - 1) / sms;
+    p.rows_per_cta = (int)std::max<int64_t>(CU_BOX_ROWS, round_up(per, CU_BOX_ROWS));
+    p.grid = (int)((b + p.rows_per_cta - 1) / p.rows_per_cta);
+    p.smem_bytes = 1024 + (size_t)p.stages * p.stage_bytes + (size_t)2 * k * 4 + 256;
+    return p;
+}
+
+template <int MT>
+__global__ void __launch_bounds__(CU_THREADS, 1)
+compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
+                     int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
+                     int tmem_cols, int rows_per_cta, const float* __restrict__ c_invnorm,
+                     int32_t* __restrict__ f, float* __restrict__ alpha) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    float* s_inv = reinterpret_cast<float*>(tiles + (size_t)stages * stage_bytes);   // [0,k) 1/||C||, [k,2k) 1/||C||^2
+
+    const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int64_t r1 = min(b, r0 + (int64_t)rows_per_cta);
+    const int ksteps = (n + CU_BLOCK_K - 1) / CU_BLOCK_K;
+    const int super_rows = MT * CU_TILE_M;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&s_empty[s], 1); }
+        for (int u = 0; u < 2; ++u) { ptx::mbar_init(&s_tfull[u], 1); ptx::mbar_init(&s_tempty[u], 4); }
+        s_abort = 0;
+        ptx::fence_barrier_init();
+        ptx::fence_proxy_async();
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&s_tmem_base, (uint32_t)tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    for (int j = threadIdx.x; j < 2 * k; j += CU_THREADS) s_inv[j] = c_invnorm[j];
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int* abort_flag = &s_abort;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (ptx::elect_one()) {
+            ptx::prefetch_tensormap(&tm_x);
+            ptx::prefetch_tensormap(&tm_c);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t st = r0; st < r1 && ok; st += super_rows) {
+                for (int ch = 0; ch < num_chunks && ok; ++ch) {
+                    for (int ks = 0; ks < ksteps; ++ks, ++it) {
+                        const int s = it % stages;
+                        const uint32_t ph = (it / stages) & 1u;
+                        if (!ptx::mbar_wait(&s_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+                        uint8_t* stage = tiles + (size_t)s * stage_bytes;
+                        uint32_t bytes = (uint32_t)n_chunk * 128u;
+                        int boxes[MT];
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const int64_t rows = min((int64_t)CU_TILE_M, r1 - (st + (int64_t)mt * CU_TILE_M));
+                            boxes[mt] = rows > 0 ? (int)((rows + CU_BOX_ROWS - 1) / CU_BOX_ROWS) : 0;
+                            bytes += (uint32_t)boxes[mt] * (CU_BOX_ROWS * 128u);
+                        }
+                        ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt)
+                            for (int q = 0; q < boxes[mt]; ++q)
+                                ptx::tma_load_2d(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
+                                                 ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
+                                                 &s_full[s]);
+                        ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, ch * n_chunk, &s_full[s]);
+                    }
+                }
+            }
+            if (!ok) {
+                raise_status(DEV_TIMEOUT);
+                // let the copies already issued land before the CTA leaves
+                const uint32_t back = it < (uint32_t)stages ? it : (uint32_t)stages;
+                int never = 0;
+                volatile int* no_abort = &never;
+                for (uint32_t d = 1; d <= back; ++d) {
+                    const uint32_t jt = it - d;
+                    ptx::mbar_wait(&s_full[jt % stages], (jt / stages) & 1u, no_abort);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (ptx::elect_one()) {
+            const uint32_t idesc = ptx::umma_idesc_bf16(CU_TILE_M, (uint32_t)n_chunk);
+            uint32_t it = 0, unit = 0;
+            bool ok = true;
+            for (int64_t st = r0; st < r1 && ok; st += super_rows) {
+                for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
+                    const uint32_t buf = unit & 1u, uph = (unit >> 1) & 1u;
+                    if (!ptx::mbar_wait(&s_tempty[buf], uph ^ 1u, abort_flag)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t d_base = tmem_base + buf * (uint32_t)(MT * n_chunk);
+                    for (int ks = 0; ks < ksteps; ++ks, ++it) {
+                        const int s = it % stages;
+                        if (!ptx::mbar_wait(&s_full[s], (it / stages) & 1u, abort_flag)) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        const uint32_t stage_addr = ptx::smem_u32(tiles + (size_t)s * stage_bytes);
+                        const uint64_t desc_b = ptx::umma_desc_k_sw128(stage_addr + MT * CU_X_TILE_BYTES);
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            if (st + (int64_t)mt * CU_TILE_M >= r1) continue;
+                            const uint64_t desc_a = ptx::umma_desc_k_sw128(stage_addr + mt * CU_X_TILE_BYTES);
+#pragma unroll
+                            for (int kk = 0; kk < CU_BLOCK_K / 16; ++kk)   // +32 bytes along K = +2 in the address field
+                                ptx::umma_bf16(d_base + (uint32_t)(mt * n_chunk), desc_a + 2 * kk, desc_b + 2 * kk, idesc,
+                                               (ks | kk) != 0);
+                        }
+                        ptx::umma_commit(&s_empty[s]);   // frees the stage once these MMAs have read it
+                    }
+                    if (ok) ptx::umma_commit(&s_tfull[buf]);
+                }
+            }
+            if (!ok) raise_status(DEV_TIMEOUT);
+        }
+    } else {
+        // ---------------- epilogue: one row per thread ----------------
+        const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
+        const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
+        uint32_t unit = 0;
+        bool ok = true;
+        for (int64_t st = r0; st < r1 && ok; st += super_rows) {
+            float best[MT], s_best[MT];
+            int j_best[MT];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) { best[mt] = -1.f; s_best[mt] = 0.f; j_best[mt] = 0; }
+            for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
+                const uint32_t buf = unit & 1u, uph = (unit >> 1) & 1u;
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_tfull[buf], uph, abort_flag));   // warp-uniform
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_base = tmem_base + buf * (uint32_t)(MT * n_chunk) + lane_base;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    if (st + (int64_t)mt * CU_TILE_M >= r1) continue;
+                    for (int c0 = 0; c0 < n_chunk; c0 += 16) {
+                        uint32_t v[16];
+                        ptx::tmem_ld_16cols(d_base + (uint32_t)(mt * n_chunk + c0), v);
+                        ptx::tmem_ld_wait();
+                        const int jb = ch * n_chunk + c0;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int j = jb + i;
+                            if (j < k) {
+                                const float s = __uint_as_float(v[i]);
+                                const float score = fabsf(s) * s_inv[j];
+                                if (score > best[mt]) { best[mt] = score; s_best[mt] = s; j_best[mt] = j; }
+                            }
+                        }
+                    }
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
+            }
+            if (ok) {
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
+                    if (row < r1) {
+                        f[row] = j_best[mt];
+                        alpha[row] = s_best[mt] * s_inv[k + j_best[mt]];
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) raise_status(DEV_TIMEOUT);
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, (uint32_t)tmem_cols);
+    }
+}
+
+inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
+                                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, int sms,
+                                        cudaStream_t st) {
+    const CompressUmmaPlan p = compress_umma_plan(b, k, sms);
+    CUtensorMap tm_x, tm_c;
+    if (!make_tmap_bf16_sw128(&tm_x, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, CU_BOX_ROWS) ||
+        !make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)p.n_chunk))
+        return PAMM_ERR_CUDA;
+    auto kern = p.mt == 2 ? compress_umma_kernel<2> : compress_umma_kernel<1>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    kern<<<p.grid, CU_THREADS, p.smem_bytes, st>>>(tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages,
+                                                   p.stage_bytes, p.tmem_cols, p.rows_per_cta, c_invnorm, f, alpha);
+    return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
+}
+
+}  // namespace pamm

@@ -2,54 +2,57 @@
 // "B' <- alpha (.) B" and "index_add"), as a deterministic segmented reduction.
 //
 //   hist    : per block of SORT_BLK rows, a histogram of f            (integers)
-//   scan    : exclusive scans -> segment starts, per-block offsets, chunk list
+//   scan    : exclusive scans -> segment starts and per-block offsets
 //   scatter : stable counting sort of row ids by f  -> perm
-//   main    : one CTA per chunk of <= CH sorted rows (all of one segment); each
-//             thread owns 16 bytes of the dY row (coalesced 128-bit loads), sums
-//             alpha_i * dY_i over the chunk's rows in ascending row order in
-//             fp32 registers, and writes one partial row
-//   reduce  : B~[j] = sum of segment j's partial rows, ascending chunk order
+//   main    : the sorted rows are cut into equal contiguous ranges, one per CTA
+//             (a single balanced wave).  Each thread owns 16 bytes of the dY row
+//             (coalesced 128-bit loads) and sums alpha_i * dY_i over its range in
+//             ascending sorted order in fp32 registers, flushing at every segment
+//             boundary: a segment that lies wholly inside the range goes straight
+//             to B~, a segment cut by a range boundary goes to a partial row
+//   reduce  : B~[j] for the cut segments = sum of their partial rows, ascending
 //
-// dY is read exactly once; the extra traffic is the partial rows
-// (<= (b/CH + k) * m * 4 bytes written and read back).  No floating-point
-// atomics anywhere, so results are bit-reproducible.
+// dY is read exactly once; the extra traffic is at most (#CTAs + k) partial
+// rows.  No floating-point atomics anywhere, so results are bit-reproducible.
 #pragma once
 #include "pamm_common.cuh"
 
 namespace pamm {
 
-constexpr int SORT_BLK = 256;          // rows per histogram / scatter block
-constexpr int CH = 128;                // rows per chunk of the main pass
-constexpr int64_t CT_MAX_K = 49152;    // k * 4 bytes of dynamic shared memory in hist
-constexpr int CT_MAX_THREADS = 768;
-constexpr int CT_UNROLL = 4;
+constexpr int SORT_BLK = 1024;         // rows per histogram / scatter block
+constexpr int CT_TILE = 256;           // rows of (perm, alpha) staged in shared memory at a time
+constexpr int64_t CT_MAX_K = 49152;    // k * 4 bytes of dynamic shared memory in hist / scatter
+#ifndef PAMM_CT_UNROLL
+#define PAMM_CT_UNROLL 8
+#endif
+#ifndef PAMM_CT_MAX_THREADS
+#define PAMM_CT_MAX_THREADS 768
+#endif
+constexpr int CT_MAX_THREADS = PAMM_CT_MAX_THREADS;
+constexpr int CT_UNROLL = PAMM_CT_UNROLL;     // rows in flight per thread
+constexpr int CT_MAX_CTAS = 148 * 8;   // upper bound on row ranges (sizes the partial buffer)
 
 struct ContractWs {
     int32_t* hist;        // NB x k   (counts, then exclusive per-block offsets)
     int32_t* seg_start;   // k + 1
-    int32_t* chunk_base;  // k + 1
-    int32_t* chunk_seg;   // max_chunks
     int32_t* perm;        // b
-    float* partials;      // max_chunks x m_pad
+    float* partials;      // (CT_MAX_CTAS + k) x m_pad
     float* btilde;        // k x m_pad (used when the caller passes no B~)
-    int64_t nb, max_chunks, m_pad;
+    int64_t nb, m_pad;
     size_t bytes;
 };
 
 inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k) {
     ContractWs w;
     w.nb = (b + SORT_BLK - 1) / SORT_BLK;
-    w.max_chunks = (b + CH - 1) / CH + k;
     w.m_pad = round_up(m, 4);
     char* p = (char*)base;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 256); return p ? p + o : (char*)0; };
     w.hist = (int32_t*)take((size_t)w.nb * k * 4);
     w.seg_start = (int32_t*)take((size_t)(k + 1) * 4);
-    w.chunk_base = (int32_t*)take((size_t)(k + 1) * 4);
-    w.chunk_seg = (int32_t*)take((size_t)w.max_chunks * 4);
     w.perm = (int32_t*)take((size_t)b * 4);
-    w.partials = (float*)take((size_t)w.max_chunks * w.m_pad * 4);
+    w.partials = (float*)take((size_t)(CT_MAX_CTAS + k) * w.m_pad * 4);
     w.btilde = (float*)take((size_t)k * w.m_pad * 4);
     w.bytes = off;
     return w;
@@ -73,16 +76,14 @@ contract_hist_kernel(const int32_t* __restrict__ f, int64_t b, int k, int32_t* _
 
 constexpr int SCAN_THREADS = 1024;
 
-// Single CTA.  Turns the per-block counts into exclusive per-block offsets,
-// scans segment sizes into seg_start and chunk counts into chunk_base, and
-// lists the owning segment of every chunk.
+// Single CTA.  Turns the per-block counts into exclusive per-block offsets and
+// scans the segment sizes into seg_start[0..k].
 __global__ void __launch_bounds__(SCAN_THREADS)
-contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restrict__ seg_start,
-                     int32_t* __restrict__ chunk_base, int32_t* __restrict__ chunk_seg) {
-    __shared__ int32_t s_warp_a[32], s_warp_b[32];
-    __shared__ int32_t s_carry_a, s_carry_b;
+contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restrict__ seg_start) {
+    __shared__ int32_t s_warp[32];
+    __shared__ int32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) { s_carry_a = 0; s_carry_b = 0; }
+    if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < k; j0 += SCAN_THREADS) {
         const int j = j0 + tid;
@@ -90,132 +91,213 @@ contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restr
         if (j < k) {
             int32_t run = 0;
             for (int blk = 0; blk < nb; ++blk) {
-                int32_t c = hist[(int64_t)blk * k + j];
+                const int32_t c = hist[(int64_t)blk * k + j];
                 hist[(int64_t)blk * k + j] = run;
                 run += c;
             }
             cnt = run;
         }
-        const int32_t nch = (cnt + CH - 1) / CH;
-        // inclusive scan of (cnt, nch) across the CTA
-        int32_t a = cnt, c = nch;
+        int32_t a = cnt;   // inclusive scan across the CTA
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            int32_t ta = __shfl_up_sync(0xffffffffu, a, off), tc = __shfl_up_sync(0xffffffffu, c, off);
-            if (lane >= off) { a += ta; c += tc; }
+            const int32_t t = __shfl_up_sync(0xffffffffu, a, off);
+            if (lane >= off) a += t;
         }
-        if (lane == 31) { s_warp_a[warp] = a; s_warp_b[warp] = c; }
+        if (lane == 31) s_warp[warp] = a;
         __syncthreads();
         if (warp == 0) {
-            int32_t wa = s_warp_a[lane], wc = s_warp_b[lane];
+            int32_t wa = s_warp[lane];
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                int32_t ta = __shfl_up_sync(0xffffffffu, wa, off), tc = __shfl_up_sync(0xffffffffu, wc, off);
-                if (lane >= off) { wa += ta; wc += tc; }
+                const int32_t t = __shfl_up_sync(0xffffffffu, wa, off);
+                if (lane >= off) wa += t;
             }
-            s_warp_a[lane] = wa;
-            s_warp_b[lane] = wc;
+            s_warp[lane] = wa;
         }
         __syncthreads();
-        const int32_t base_a = s_carry_a + (warp ? s_warp_a[warp - 1] : 0);
-        const int32_t base_b = s_carry_b + (warp ? s_warp_b[warp - 1] : 0);
-        const int32_t excl_a = base_a + a - cnt, excl_b = base_b + c - nch;
-        if (j < k) {
-            seg_start[j] = excl_a;
-            chunk_base[j] = excl_b;
-            for (int32_t w = 0; w < nch; ++w) chunk_seg[excl_b + w] = j;
-        }
+        const int32_t base = s_carry + (warp ? s_warp[warp - 1] : 0);
+        if (j < k) seg_start[j] = base + a - cnt;
         __syncthreads();
-        if (tid == SCAN_THREADS - 1) { s_carry_a = base_a + a; s_carry_b = base_b + c; }
+        if (tid == SCAN_THREADS - 1) s_carry = base + a;
         __syncthreads();
     }
-    if (tid == 0) { seg_start[k] = s_carry_a; chunk_base[k] = s_carry_b; }
+    if (tid == 0) seg_start[k] = s_carry;
 }
 
+// Stable scatter: rows of one block are ranked warp by warp (ascending row
+// order); inside a warp, match_any groups equal keys and the lowest lane of a
+// group reserves the group's slots.
 __global__ void __launch_bounds__(SORT_BLK)
 contract_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const int32_t* __restrict__ hist,
                         const int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
-    __shared__ int32_t s_f[SORT_BLK];
-    const int tid = threadIdx.x;
+    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t* my_hist = hist + (int64_t)blockIdx.x * k;
+    for (int j = tid; j < k; j += SORT_BLK) s_next[j] = seg_start[j] + my_hist[j];
     const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
     int32_t j = -1;
     if (i < b) {
         j = f[i];
         if (j < 0 || j >= k) j = -1;
     }
-    s_f[tid] = j;
-    __syncthreads();
-    if (j < 0) return;
-    int rank = 0;
-    for (int t = 0; t < tid; ++t) rank += (s_f[t] == j);
-    perm[seg_start[j] + hist[(int64_t)blockIdx.x * k + j] + rank] = (int32_t)i;
+    const unsigned peers = __match_any_sync(0xffffffffu, j);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    const int leader = __ffs(peers) - 1;
+    const int count = __popc(peers);
+    for (int w = 0; w < SORT_BLK / 32; ++w) {
+        __syncthreads();
+        if (warp == w) {
+            int32_t base = 0;
+            if (lane == leader && j >= 0) {
+                base = s_next[j];
+                s_next[j] = base + count;
+            }
+            base = __shfl_sync(0xffffffffu, base, leader);
+            if (j >= 0) perm[base + rank] = (int32_t)i;
+        }
+    }
+}
+
+// First index j in [0,k) with seg_start[j] <= r < seg_start[j+1].
+__device__ __forceinline__ int segment_of(const int32_t* __restrict__ seg_start, int k, int32_t r) {
+    int lo = 0, hi = k;   // invariant: seg_start[lo] <= r < seg_start[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (seg_start[mid] <= r) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// acc += a * (16 bytes of T held in raw)
+template <typename T>
+__device__ __forceinline__ void fma_raw(float (&acc)[Vec16<T>::N], float a, const uint4& raw);
+template <>
+__device__ __forceinline__ void fma_raw<float>(float (&acc)[4], float a, const uint4& raw) {
+    acc[0] = fmaf(a, __uint_as_float(raw.x), acc[0]); acc[1] = fmaf(a, __uint_as_float(raw.y), acc[1]);
+    acc[2] = fmaf(a, __uint_as_float(raw.z), acc[2]); acc[3] = fmaf(a, __uint_as_float(raw.w), acc[3]);
+}
+template <>
+__device__ __forceinline__ void fma_raw<__nv_bfloat16>(float (&acc)[8], float a, const uint4& raw) {
+    acc[0] = fmaf(a, bf16_lo(raw.x), acc[0]); acc[1] = fmaf(a, bf16_hi(raw.x), acc[1]);
+    acc[2] = fmaf(a, bf16_lo(raw.y), acc[2]); acc[3] = fmaf(a, bf16_hi(raw.y), acc[3]);
+    acc[4] = fmaf(a, bf16_lo(raw.z), acc[4]); acc[5] = fmaf(a, bf16_hi(raw.z), acc[5]);
+    acc[6] = fmaf(a, bf16_lo(raw.w), acc[6]); acc[7] = fmaf(a, bf16_hi(raw.w), acc[7]);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(CT_MAX_THREADS)
 contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, int64_t ldy, int64_t m,
-                     int k, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ chunk_base,
-                     const int32_t* __restrict__ chunk_seg, const int32_t* __restrict__ perm,
-                     float* __restrict__ partials, int64_t m_pad) {
+                     int k, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ perm,
+                     int rows_per_cta, float* __restrict__ partials, int64_t m_pad,
+                     float* __restrict__ Bt, int64_t ldb) {
     constexpr int V = Vec16<T>::N;
-    __shared__ int32_t s_row[CH];
-    __shared__ float s_alpha[CH];
-    const int w = blockIdx.x;
-    if (w >= chunk_base[k]) return;
-    const int j = chunk_seg[w];
-    const int r0 = seg_start[j] + (w - chunk_base[j]) * CH;
-    const int cnt = min(CH, seg_start[j + 1] - r0);
-    for (int t = threadIdx.x; t < cnt; t += blockDim.x) {
-        const int32_t i = perm[r0 + t];
-        s_row[t] = i;
-        s_alpha[t] = alpha[i];
-    }
-    __syncthreads();
+    __shared__ int32_t s_row[CT_TILE];
+    __shared__ float s_alpha[CT_TILE];
+    const int c = blockIdx.x;
+    const int32_t total = seg_start[k];
+    const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
+    const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
+    if (r_begin >= r_end) return;
     const int64_t col = ((int64_t)blockIdx.y * blockDim.x + threadIdx.x) * V;
-    if (col >= m) return;
+    const bool active = col < m;
+    const bool full_vec = col + V <= m;
+    int j = segment_of(seg_start, k, r_begin);
+    int32_t j_end = seg_start[j + 1];
+
     float acc[V];
 #pragma unroll
     for (int e = 0; e < V; ++e) acc[e] = 0.f;
-    int t = 0;
-    for (; t + CT_UNROLL <= cnt; t += CT_UNROLL) {
-        float x[CT_UNROLL][V];
+
+    auto flush = [&](int seg) {
+        if (!active) return;
+        const bool inside = seg_start[seg] >= r_begin && seg_start[seg + 1] <= r_end;
+        if (inside) {
+            float* out = Bt + (int64_t)seg * ldb + col;
 #pragma unroll
-        for (int u = 0; u < CT_UNROLL; ++u) load_vec<T>(dY + (int64_t)s_row[t + u] * ldy, col, m, x[u]);
+            for (int e = 0; e < V; e += 4) {
+                if (col + e + 4 <= m) {
+                    *reinterpret_cast<float4*>(out + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+                } else {
+                    for (int t = 0; t < 4 && col + e + t < m; ++t) out[e + t] = acc[e + t];
+                }
+            }
+        } else {
+            float* out = partials + (int64_t)(c + seg) * m_pad + col;   // m_pad % 4 == 0, col % V == 0
 #pragma unroll
-        for (int u = 0; u < CT_UNROLL; ++u) {
-            const float a = s_alpha[t + u];
-#pragma unroll
-            for (int e = 0; e < V; ++e) acc[e] = fmaf(a, x[u][e], acc[e]);
+            for (int e = 0; e < V; e += 4)
+                if (col + e < m_pad) *reinterpret_cast<float4*>(out + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
         }
-    }
-    for (; t < cnt; ++t) {
-        float x[V];
-        load_vec<T>(dY + (int64_t)s_row[t] * ldy, col, m, x);
-        const float a = s_alpha[t];
+    };
+
+    for (int32_t t0 = r_begin; t0 < r_end; t0 += CT_TILE) {
+        const int tcnt = min(CT_TILE, r_end - t0);
+        __syncthreads();
+        for (int t = threadIdx.x; t < tcnt; t += blockDim.x) {
+            const int32_t i = perm[t0 + t];
+            s_row[t] = i;
+            s_alpha[t] = alpha[i];
+        }
+        __syncthreads();
+        int pos = 0;
+        while (pos < tcnt) {
+            const int lim = min(tcnt, j_end - t0);
+            if (active && full_vec) {
+                int t = pos;
+                for (; t + CT_UNROLL <= lim; t += CT_UNROLL) {
+                    uint4 raw[CT_UNROLL];
 #pragma unroll
-        for (int e = 0; e < V; ++e) acc[e] = fmaf(a, x[e], acc[e]);
-    }
-    float* out = partials + (int64_t)w * m_pad + col;   // m_pad is a multiple of 4, col of V
+                    for (int u = 0; u < CT_UNROLL; ++u)
+                        raw[u] = __ldg(reinterpret_cast<const uint4*>(dY + (int64_t)s_row[t + u] * ldy + col));
 #pragma unroll
-    for (int e = 0; e < V; e += 4)
-        if (col + e < m_pad) *reinterpret_cast<float4*>(out + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+                    for (int u = 0; u < CT_UNROLL; ++u) fma_raw<T>(acc, s_alpha[t + u], raw[u]);
+                }
+                for (; t < lim; ++t)
+                    fma_raw<T>(acc, s_alpha[t], __ldg(reinterpret_cast<const uint4*>(dY + (int64_t)s_row[t] * ldy + col)));
+            } else if (active) {   // ragged last vector of the row
+                for (int t = pos; t < lim; ++t) {
+                    float x[V];
+                    load_vec<T>(dY + (int64_t)s_row[t] * ldy, col, m, x);
+                    const float a = s_alpha[t];
+#pragma unroll
+                    for (int e = 0; e < V; ++e) acc[e] = fmaf(a, x[e], acc[e]);
+                }
+            }
+            pos = lim;
+            if (t0 + pos == j_end) {          // segment j is complete
+                flush(j);
+#pragma unroll
+                for (int e = 0; e < V; ++e) acc[e] = 0.f;
+                if (j_end >= r_end) { j = -1; break; }
+                do { ++j; j_end = seg_start[j + 1]; } while (j_end <= t0 + pos);   // skip empty segments
+            }
+        }
+        if (j < 0) break;
+    }
+    if (j >= 0) flush(j);   // the range ended inside segment j
 }
 
 constexpr int RED_THREADS = 256;
 
+// Finishes B~: zero rows for empty segments, sums of partial rows for segments
+// that were cut by a range boundary; rows written directly by main are left alone.
 __global__ void __launch_bounds__(RED_THREADS)
 contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k,
-                       const int32_t* __restrict__ chunk_base, float* __restrict__ Bt, int64_t ldb) {
+                       const int32_t* __restrict__ seg_start, int rows_per_cta,
+                       float* __restrict__ Bt, int64_t ldb) {
     const int64_t mv = m_pad / 4;
     const int64_t idx = (int64_t)blockIdx.x * RED_THREADS + threadIdx.x;
     if (idx >= (int64_t)k * mv) return;
     const int j = (int)(idx / mv);
     const int64_t col = (idx % mv) * 4;
-    const int w0 = chunk_base[j], w1 = chunk_base[j + 1];
+    const int32_t s0 = seg_start[j], s1 = seg_start[j + 1];
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int w = w0; w < w1; ++w) {
-        const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)w * m_pad + col);
-        s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+    if (s1 > s0) {
+        const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;
+        if (c_lo == c_hi) return;
+        for (int c = c_lo; c <= c_hi; ++c) {
+            const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)(c + j) * m_pad + col);
+            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+        }
     }
     float* out = Bt + (int64_t)j * ldb + col;
     if (col + 4 <= m) {

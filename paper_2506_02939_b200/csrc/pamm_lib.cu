@@ -97,29 +97,48 @@ pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t 
     return launch_status();
 }
 
+int sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            sms = 148;
+    }
+    return sms;
+}
+
 template <typename T>
 pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
                             int64_t k, float* Bt, int64_t ldb, const ContractWs& w, cudaStream_t st) {
     constexpr int V = Vec16<T>::N;
     const size_t hsmem = (size_t)k * 4;
     if (hsmem > 48 * 1024 &&
-        cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess)
+        (cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess ||
+         cudaFuncSetAttribute(contract_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess))
         return PAMM_ERR_CUDA;
     contract_hist_kernel<<<(int)w.nb, SORT_BLK, hsmem, st>>>(f, b, (int)k, w.hist);
-    contract_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(w.hist, (int)w.nb, (int)k, w.seg_start, w.chunk_base, w.chunk_seg);
-    contract_scatter_kernel<<<(int)w.nb, SORT_BLK, 0, st>>>(f, b, (int)k, w.hist, w.seg_start, w.perm);
+    contract_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(w.hist, (int)w.nb, (int)k, w.seg_start);
+    contract_scatter_kernel<<<(int)w.nb, SORT_BLK, hsmem, st>>>(f, b, (int)k, w.hist, w.seg_start, w.perm);
+    // one balanced wave: every CTA gets the same number of sorted rows
     const int64_t vecs = (m + V - 1) / V;
     const int64_t slabs = (vecs + CT_MAX_THREADS - 1) / CT_MAX_THREADS;
     const int threads = (int)round_up((vecs + slabs - 1) / slabs, 32);
-    dim3 grid((unsigned)w.max_chunks, (unsigned)slabs);
+    int occ = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, contract_main_kernel<T>, threads, 0) != cudaSuccess || occ < 1)
+        occ = 1;
+    int64_t ranges = std::max<int64_t>(1, std::min<int64_t>(CT_MAX_CTAS, (int64_t)sm_count() * occ / slabs));
+    const int64_t rows_per_cta = std::max<int64_t>(32, (b + ranges - 1) / ranges);
+    ranges = (b + rows_per_cta - 1) / rows_per_cta;
+    dim3 grid((unsigned)ranges, (unsigned)slabs);
     prof_begin(PAMM_PROF_CONTRACT, st);
-    contract_main_kernel<T><<<grid, threads, 0, st>>>(alpha, (const T*)dY, ldy, m, (int)k, w.seg_start, w.chunk_base,
-                                                      w.chunk_seg, w.perm, w.partials, w.m_pad);
+    contract_main_kernel<T><<<grid, threads, 0, st>>>(alpha, (const T*)dY, ldy, m, (int)k, w.seg_start, w.perm,
+                                                      (int)rows_per_cta, w.partials, w.m_pad, Bt, ldb);
     prof_end(PAMM_PROF_CONTRACT, st);
-    g_launches += 5;
     const int64_t items = k * (w.m_pad / 4);
     contract_reduce_kernel<<<(int)((items + RED_THREADS - 1) / RED_THREADS), RED_THREADS, 0, st>>>(
-        w.partials, w.m_pad, m, (int)k, w.chunk_base, Bt, ldb);
+        w.partials, w.m_pad, m, (int)k, w.seg_start, (int)rows_per_cta, Bt, ldb);
+    g_launches += 5;
     return launch_status();
 }
 
@@ -184,8 +203,13 @@ pamm_status check_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, 
 pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
                         int64_t k, const float* c_invnorm, int32_t* f, float* alpha, cudaStream_t st) {
     if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
-    if (compress_umma_supported(b, n, k))
-        return launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+    if (compress_umma_supported(b, n, k)) {
+        prof_begin(PAMM_PROF_COMPRESS, st);
+        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), st);
+        prof_end(PAMM_PROF_COMPRESS, st);
+        g_launches += 1;
+        return s;
+    }
     return launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
 }
 

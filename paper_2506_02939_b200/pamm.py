@@ -11,7 +11,10 @@ from pathlib import Path
 
 import torch
 
-_LIB_PATH = Path(__file__).resolve().parent / "libpamm_b200.so"
+import os
+
+# PAMM_B200_LIB points the binding at another build of the same library (tuning builds).
+_LIB_PATH = Path(os.environ.get("PAMM_B200_LIB") or Path(__file__).resolve().parent / "libpamm_b200.so")
 if not _LIB_PATH.exists():
     raise ImportError(
         f"{_LIB_PATH} is missing: build it with `python -m paper_2506_02939_b200.build` "
@@ -89,6 +92,13 @@ def _stream(stream) -> ctypes.c_void_p:
     return ctypes.c_void_p(s.cuda_stream)
 
 
+def alloc_matrix(rows: int, cols: int, dtype, device="cuda") -> torch.Tensor:
+    """rows x cols view whose row stride is padded so that every row starts 16-byte aligned."""
+    per = 16 // torch.empty((), dtype=dtype).element_size()
+    ld = (cols + per - 1) // per * per
+    return torch.empty((rows, ld), dtype=dtype, device=device)[:, :cols]
+
+
 def workspace_bytes(kind: int, b: int, n: int, m: int, k: int, dtype: int) -> int:
     r = _lib.pamm_workspace_bytes(kind, b, n, m, k, dtype)
     if r == ctypes.c_size_t(-1).value:
@@ -109,7 +119,7 @@ def draw_indices_host(b: int, k: int, seed: int) -> torch.Tensor:
 def select_generators(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, stream=None):
     b, n = X.shape
     idx_out = torch.empty(k, dtype=torch.int32, device=X.device) if idx_out is None else idx_out
-    C = torch.empty((k, n), dtype=X.dtype, device=X.device) if C is None else C
+    C = alloc_matrix(k, n, X.dtype, X.device) if C is None else C
     c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=X.device) if c_invnorm is None else c_invnorm
     _check(_lib.pamm_select_generators(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out),
                                        _ptr(C), _ld(C), _ptr(c_invnorm), _stream(stream)), "pamm_select_generators")
@@ -132,7 +142,7 @@ def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, 
     b, n = X.shape
     dev = X.device
     idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
-    C = torch.empty((k, n), dtype=X.dtype, device=dev) if C is None else C
+    C = alloc_matrix(k, n, X.dtype, dev) if C is None else C
     c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
     f = torch.empty(b, dtype=torch.int32, device=dev) if f is None else f
     alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
@@ -145,7 +155,7 @@ def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, 
 
 def contract(f, alpha, dY, k: int, Btilde=None, workspace=None, stream=None):
     b, m = dY.shape
-    Btilde = torch.empty((k, m), dtype=torch.float32, device=dY.device) if Btilde is None else Btilde
+    Btilde = alloc_matrix(k, m, torch.float32, dY.device) if Btilde is None else Btilde
     if workspace is None:
         workspace = alloc_workspace(WS_CONTRACT, b, 1, m, k, _dt(dY), dY.device)
     _check(_lib.pamm_contract(_ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde), _ld(Btilde),
@@ -156,7 +166,7 @@ def contract(f, alpha, dY, k: int, Btilde=None, workspace=None, stream=None):
 def weight_grad(C, Btilde, dW=None, stream=None):
     k, n = C.shape
     m = Btilde.shape[1]
-    dW = torch.empty((n, m), dtype=torch.float32, device=C.device) if dW is None else dW
+    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
     _check(_lib.pamm_weight_grad(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW),
                                  _stream(stream)), "pamm_weight_grad")
     return dW
@@ -165,7 +175,7 @@ def weight_grad(C, Btilde, dW=None, stream=None):
 def contract_weight_grad(C, f, alpha, dY, Btilde=None, dW=None, workspace=None, stream=None):
     k, n = C.shape
     b, m = dY.shape
-    dW = torch.empty((n, m), dtype=torch.float32, device=C.device) if dW is None else dW
+    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
     if workspace is None:
         workspace = alloc_workspace(WS_CONTRACT, b, n, m, k, _dt(dY), dY.device)
     _check(_lib.pamm_contract_weight_grad(_ptr(C), _ld(C), n, _ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY),

@@ -102,7 +102,8 @@ def run_and_compare(X: np.ndarray, dY: np.ndarray, k: int, seed: int = 0, idx_in
     # ---- GPU ------------------------------------------------------------------
     if fused:
         idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, seed, idx_in=idx_d)
-        Bt = torch.full((k, m), float("nan"), dtype=torch.float32, device="cuda")
+        Bt = pamm.alloc_matrix(k, m, torch.float32)
+        Bt.fill_(float("nan"))
         dW = pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt)
     else:
         idx, C, invn = pamm.select_generators(Xd, k, seed, idx_in=idx_d)

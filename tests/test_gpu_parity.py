@@ -175,7 +175,7 @@ def test_unfused_stage_inputs_from_elsewhere():
     f = rng.integers(0, k, size=b).astype(np.int32)
     f[f == 4] = 5                                                     # an empty segment
     a = rng.standard_normal(b).astype(np.float32)
-    Bt = pamm.contract(torch.from_numpy(f).cuda(), torch.from_numpy(a).cuda(), parity.to_device(dY), k)
+    Bt = pamm.contract(torch.from_numpy(f).cuda(), torch.from_numpy(a).cuda(), parity.to_device(dY, ld=304), k)
     ref = orc.contract(f, a.astype(np.float64), dY, k)
     assert parity.rel_fro(Bt.cpu().numpy(), ref) <= 1e-5
     assert torch.all(Bt[4] == 0)
