@@ -216,8 +216,13 @@ pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_d
 pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
                            int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
     if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
-    if (weight_grad_mma_supported(k, n, m))
-        return launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+    if (weight_grad_mma_supported(k, n, m)) {
+        prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
+        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+        prof_end(PAMM_PROF_WEIGHT_GRAD, st);
+        g_launches += 1;
+        return s;
+    }
     return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
 }
 
