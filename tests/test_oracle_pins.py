@@ -66,7 +66,7 @@ def test_generators_represent_themselves():
     f, alpha, t1, _ = orc.compress(X, C, q)
     assert np.array_equal(C, synth.to_f64(X)[I])
     assert np.array_equal(f[I], np.arange(len(I)))
-    # alpha = <C_j,C_j>/||C_j||^2 = 1 (Appendix B: "A_i can always generate itself with alpha=1")
+    # alpha = <C_j,C_j>/||C_j||^2 = 1 (proof of Lemma 2: a row can always generate itself with alpha = 1)
     assert np.all(alpha[I] == 1.0)
     d = brute_force_assignment(synth.to_f64(X)[I], C)
     assert np.allclose(np.diag(d), 0.0, atol=1e-12)
@@ -83,7 +83,7 @@ def test_residual_orthogonal_and_identity():
     dots = np.einsum("il,il->i", R, C[f])
     scale = np.linalg.norm(X64, axis=1) * np.linalg.norm(C[f], axis=1)
     assert np.all(np.abs(dots) <= 1e-12 * scale)
-    # ||A_i - A~_i||^2 = ||A_i||^2 (1 - csim^2)   (Appendix A, with the square restored)
+    # ||A_i - A~_i||^2 = ||A_i||^2 (1 - csim^2)   (proof of Lemma 1, with the square restored)
     csim = np.einsum("il,il->i", X64, C[f]) / scale
     lhs = np.sum(R * R, axis=1)
     rhs = np.sum(X64 * X64, axis=1) * (1 - csim ** 2)
@@ -293,7 +293,7 @@ def test_paper_printed_values():
 
 
 def test_clustered_data_error_decreases_with_k():
-    """Qualitative claim of Appendix F: E(r) falls as k grows (here on clustered synthetic rows)."""
+    """Qualitative claim of the appendix "PAMM Compression EDA": E(r) falls as k grows (here on clustered synthetic rows)."""
     X, dY = synth.random_case(512, 32, 16, "f32", 24, centres=8, noise=0.05)
     exact = X.astype(np.float64).T @ dY.astype(np.float64)
     errs = []
