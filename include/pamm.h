@@ -175,6 +175,43 @@ pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host,
                                void* arena, size_t arena_bytes, void* stream);
 
 /*
+ * Contract without any caller-provided or library-allocated scratch (the paper
+ * has no counterpart: this entry exists for the benefit of some callers, not
+ * for the method).  It computes exactly what pamm_contract computes, with the
+ * same kernels, but its scratch is a fixed array of PAMM_NO_ALLOC_SCRATCH_BYTES
+ * that is part of the library image, so nothing is allocated or freed by this
+ * call: no cudaMalloc / cudaFree, no allocating library routine.
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the
+ * point where it needs B~ -- a plugin running inside a host application that
+ * owns the whole memory budget, a step running between the stages of a
+ * latency-critical loop where cudaMalloc's implicit device synchronisation is
+ * unacceptable, or a callback that runs while the framework's allocator is
+ * locked.  Such a caller still owns f, alpha, dY and Btilde and passes them in.
+ *
+ * Limits and sharing:
+ *  - the problem must be small enough for the fixed array:
+ *    pamm_workspace_bytes(PAMM_WS_CONTRACT, b, n, m, k, dt) must not exceed
+ *    PAMM_NO_ALLOC_SCRATCH_BYTES, otherwise PAMM_ERR_WORKSPACE is returned and
+ *    nothing is launched;
+ *  - every device that loads the library holds the array until the process
+ *    exits, whether or not this entry is ever called;
+ *  - the first call on a device looks up the array's device address (once per
+ *    device, with that device current) before it launches anything; make that
+ *    first call outside any stream capture;
+ *  - all calls on one device share the one array and find in it whatever the
+ *    previous call left.  The kernels write every word of it before they read
+ *    it, so nothing has to be cleared between calls, but two calls that overlap
+ *    on the GPU (different streams, no ordering between them) race on it and
+ *    give wrong results.  Calls on one stream are ordered and safe.
+ * Arguments, layout and error behaviour are those of pamm_contract.
+ */
+#define PAMM_NO_ALLOC_SCRATCH_BYTES (8u << 20)
+pamm_status pamm_contract_no_alloc(const int32_t* f, const float* alpha, const void* dY, int64_t ldy,
+                                   int64_t b, int64_t m, pamm_dtype dt, int64_t k,
+                                   float* Btilde, int64_t ldb, void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the current device's status
  * word.  Returns PAMM_OK, PAMM_ERR_TIMEOUT, PAMM_ERR_BAD_INDEX, or
  * PAMM_ERR_CUDA if the stream itself reports an error.

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "pamm_common.cuh"
@@ -390,3 +391,46 @@ pamm_status pamm_last_device_status(void* stream) {
 }
 
 }  // extern "C"
+
+// ---- scratch of pamm_contract_no_alloc -----------------------------------------
+// Lives in the library image, one copy per device that loads it.  In host code
+// the name below is only a stand-in for the symbol: the device address has to be
+// asked for with cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_no_alloc_scratch[PAMM_NO_ALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int NO_ALLOC_MAX_DEVICES = 64;
+void* g_no_alloc_ptr[NO_ALLOC_MAX_DEVICES] = {};
+std::mutex g_no_alloc_mutex;
+
+// Device address of the fixed scratch on the current device (nullptr on failure).
+void* no_alloc_scratch_ptr() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NO_ALLOC_MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_no_alloc_mutex);
+    if (!g_no_alloc_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_no_alloc_scratch) != cudaSuccess || !p) return nullptr;
+        g_no_alloc_ptr[dev] = p;
+    }
+    return g_no_alloc_ptr[dev];
+}
+}  // namespace
+
+extern "C" pamm_status pamm_contract_no_alloc(const int32_t* f, const float* alpha, const void* dY, int64_t ldy,
+                                              int64_t b, int64_t m, pamm_dtype dt, int64_t k, float* Btilde,
+                                              int64_t ldb, void* stream) {
+    // sizes first: the fixed array is the only scratch there is
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (b < 1 || m < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (contract_ws_layout(nullptr, b, m, k).bytes > (size_t)PAMM_NO_ALLOC_SCRATCH_BYTES) return PAMM_ERR_WORKSPACE;
+    void* scratch = no_alloc_scratch_ptr();
+    if (!scratch) return PAMM_ERR_CUDA;
+    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, scratch,
+                                   (size_t)PAMM_NO_ALLOC_SCRATCH_BYTES);
+    if (s != PAMM_OK) return s;
+    const ContractWs w = contract_ws_layout(scratch, b, m, k);
+    cudaStream_t st = (cudaStream_t)stream;
+    return dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st)
+                          : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st);
+}

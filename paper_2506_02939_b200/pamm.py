@@ -39,6 +39,7 @@ _SIGNATURES = {
     "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
     "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
     "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
     "pamm_last_device_status": ([_vp], _ci),
     "pamm_launch_count": ([], ctypes.c_ulonglong),
     "pamm_set_profile_events": ([_ci, _vp, _vp], _ci),
@@ -160,6 +161,22 @@ def contract(f, alpha, dY, k: int, Btilde=None, workspace=None, stream=None):
         workspace = alloc_workspace(WS_CONTRACT, b, 1, m, k, _dt(dY), dY.device)
     _check(_lib.pamm_contract(_ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde), _ld(Btilde),
                               _ptr(workspace), workspace.numel(), _stream(stream)), "pamm_contract")
+    return Btilde
+
+
+NO_ALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def contract_no_alloc(f, alpha, dY, k: int, Btilde, stream=None):
+    """``contract`` for callers that may not allocate device memory where they need B~ (a plugin inside a host
+    application that owns the memory budget, a latency-critical loop that cannot afford cudaMalloc's device
+    synchronisation, a callback running while the framework's allocator is locked).  The scratch is a fixed
+    8 MiB array inside the library, shared by every call on the device: keep calls on one stream (overlapping
+    calls race on it), make the first call on a device outside stream capture, and pass ``Btilde`` yourself --
+    this wrapper allocates nothing either.  Problems whose scratch would not fit raise ``ERR_WORKSPACE``."""
+    b, m = dY.shape
+    _check(_lib.pamm_contract_no_alloc(_ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde),
+                                       _ld(Btilde), _stream(stream)), "pamm_contract_no_alloc")
     return Btilde
 
 
