@@ -29,6 +29,7 @@ if str(ROOT) not in sys.path:
 
 METRIC = "PAMM compress + weight-grad tokens/sec per QKV layer; achieved HBM GB/s vs peak"
 FALLBACK_HBM_GBS = 6650.0
+PROF_EVERY = 4      # steps between two steps that carry per-kernel CUDA events
 # DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
 # summarised under profiles/, keyed by workload; None until captured.
 NCU_TRAFFIC_BYTES = {}
@@ -83,7 +84,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(self.gpu)],
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i", str(self.gpu)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -145,14 +146,27 @@ def run_reference(args):
     from paper_2506_02939_b200 import synth
     w = synth.WORKLOADS[args.workload]
     k = w.ks[0]
-    seqs = max(1, min(w.num_seqs, args.ref_tokens // w.seq_len))
-    inp = synth.make_inputs(args.workload, num_seqs=seqs)
-    b = inp.b
-    rng = np.random.default_rng(w.index_seed)
-    I = np.sort(rng.choice(b, size=min(k, b), replace=False)).astype(np.int32)
+    max_seqs = max(1, min(w.num_seqs, args.ref_tokens // w.seq_len))
+    full = synth.make_inputs(args.workload, num_seqs=max_seqs)
+
+    def sample(seqs):
+        bs = seqs * w.seq_len
+        rng = np.random.default_rng(w.index_seed)
+        return full.X[:bs], full.dY[:bs], np.sort(rng.choice(bs, size=min(k, bs), replace=False)).astype(np.int32)
+
+    # size the per-step sample so that all steps fit the time budget: one calibration pass on one sequence
+    Xc, dYc, Ic = sample(1)
+    orc.pamm(Xc, Ic, dYc)
+    t0 = time.perf_counter()
+    orc.pamm(Xc, Ic, dYc)
+    per_seq = max(1e-6, time.perf_counter() - t0)
+    seqs = int(args.ref_budget_s / (max(1, args.steps + args.warmup) * per_seq))
+    seqs = max(1, min(max_seqs, seqs))
+    X, dY, I = sample(seqs)
+    b = X.shape[0]
 
     def step():
-        orc.pamm(inp.X, I, inp.dY)
+        orc.pamm(X, I, dY)
 
     for _ in range(args.warmup):
         step()
@@ -226,7 +240,10 @@ def run_cuda(args):
     # ---- timed region: device-resident inputs ----------------------------------
     K = args.steps
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    kev = {kind: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    # per-kernel event pairs on every PROF_EVERY-th step only: an event between two
+    # kernels serialises them, the other steps keep the back-to-back launch overlap
+    prof_steps = [s for s in range(K) if s % PROF_EVERY == 0]
+    kev = {kind: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in prof_steps]
            for kind in (pamm.PROF_COMPRESS, pamm.PROF_CONTRACT, pamm.PROF_WEIGHT_GRAD)}
     for kind in kev:                       # create the underlying CUDA events
         for a, z in kev[kind]:
@@ -240,8 +257,12 @@ def run_cuda(args):
     sampler.start()
     t_begin.record(stream)
     for s in range(K):
-        for kind in kev:
-            pamm.set_profile_events(kind, kev[kind][s][0], kev[kind][s][1])
+        if s % PROF_EVERY == 0:
+            for kind in kev:
+                pamm.set_profile_events(kind, kev[kind][s // PROF_EVERY][0], kev[kind][s // PROF_EVERY][1])
+        elif s % PROF_EVERY == 1:
+            for kind in kev:
+                pamm.set_profile_events(kind, None, None)
         ev[s][0].record(stream)
         pamm.compress_fused(X, k, w.index_seed + s, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
         ev[s][1].record(stream)
@@ -259,8 +280,9 @@ def run_cuda(args):
         raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
     ms_total_local = t_begin.elapsed_time(t_end)
     ms_total, tokens = aggregate(ms_total_local, b * K, device=dev)
-    fwd = np.array([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)])
-    bwd = np.array([ev[s][1].elapsed_time(ev[s][2]) for s in range(K)])
+    plain = [s for s in range(K) if s % PROF_EVERY != 0] or list(range(K))
+    fwd = np.array([ev[s][0].elapsed_time(ev[s][1]) for s in plain])
+    bwd = np.array([ev[s][1].elapsed_time(ev[s][2]) for s in plain])
     kern = {kind: np.array([a.elapsed_time(z) for a, z in kev[kind]]) for kind in kev}
 
     # ---- end to end through the host-buffer entry point ----------------------------
@@ -345,12 +367,13 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="c4", help="c1..c5; c4 (LLaMA-1B-shaped) is the headline configuration")
     ap.add_argument("--k", type=int, default=0, help="override the workload's generator count")
     ap.add_argument("--ref-tokens", type=int, default=16384, help="tokens per oracle pass (bounded sample)")
+    ap.add_argument("--ref-budget-s", type=float, default=120.0, help="time budget of the whole --impl reference run")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -94,6 +94,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         ptx::tmem_alloc(&s_tmem_base, (uint32_t)tmem_cols);
         ptx::tmem_relinquish();
     }
+    grid_dependency_wait();     // C and the norms come from the kernel before
     for (int j = threadIdx.x; j < 2 * k; j += CU_THREADS) s_inv[j] = c_invnorm[j];
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -253,8 +254,18 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
     auto kern = p.mt == 2 ? compress_umma_kernel<2> : compress_umma_kernel<1>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
         return PAMM_ERR_CUDA;
-    kern<<<p.grid, CU_THREADS, p.smem_bytes, st>>>(tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages,
-                                                   p.stage_bytes, p.tmem_cols, p.rows_per_cta, c_invnorm, f, alpha);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(CU_THREADS);
+    cfg.dynamicSmemBytes = p.smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set up while the select kernel runs
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
+                       p.tmem_cols, p.rows_per_cta, c_invnorm, f, alpha);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

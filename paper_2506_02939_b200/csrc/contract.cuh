@@ -61,6 +61,7 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
 __global__ void __launch_bounds__(SORT_BLK)
 contract_hist_kernel(const int32_t* __restrict__ f, int64_t b, int k, int32_t* __restrict__ hist) {
     extern __shared__ int32_t s_hist[];
+    grid_launch_dependents();
     for (int j = threadIdx.x; j < k; j += SORT_BLK) s_hist[j] = 0;
     __syncthreads();
     const int64_t i = (int64_t)blockIdx.x * SORT_BLK + threadIdx.x;
@@ -83,6 +84,8 @@ contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restr
     __shared__ int32_t s_warp[32];
     __shared__ int32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < k; j0 += SCAN_THREADS) {
@@ -133,7 +136,91 @@ contract_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const i
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t* my_hist = hist + (int64_t)blockIdx.x * k;
+    grid_dependency_wait();
+    grid_launch_dependents();
     for (int j = tid; j < k; j += SORT_BLK) s_next[j] = seg_start[j] + my_hist[j];
+    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
+    int32_t j = -1;
+    if (i < b) {
+        j = f[i];
+        if (j < 0 || j >= k) j = -1;
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, j);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    const int leader = __ffs(peers) - 1;
+    const int count = __popc(peers);
+    for (int w = 0; w < SORT_BLK / 32; ++w) {
+        __syncthreads();
+        if (warp == w) {
+            int32_t base = 0;
+            if (lane == leader && j >= 0) {
+                base = s_next[j];
+                s_next[j] = base + count;
+            }
+            base = __shfl_sync(0xffffffffu, base, leader);
+            if (j >= 0) perm[base + rank] = (int32_t)i;
+        }
+    }
+}
+
+// Scan and scatter in one launch, for the common case of a small histogram
+// matrix: every block derives what it needs from the raw per-block counts --
+// the segment starts (an exclusive scan over j of the column totals) and its own
+// offset inside every segment (the counts of the blocks before it) -- and then
+// scatters its rows exactly as contract_scatter_kernel does.  Block 0 also
+// publishes seg_start.  Costs nb * k reads per block instead of a serial
+// single-CTA pass between two launches.
+__global__ void __launch_bounds__(SORT_BLK)
+contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const int32_t* __restrict__ hist,
+                             int nb, int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
+    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
+    __shared__ int32_t s_warp[32];
+    __shared__ int32_t s_carry;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int j0 = 0; j0 < k; j0 += SORT_BLK) {
+        const int j = j0 + tid;
+        int32_t total = 0, before = 0;
+        if (j < k) {
+            for (int blk = 0; blk < nb; ++blk) {
+                const int32_t c = __ldg(hist + (int64_t)blk * k + j);
+                before += blk < (int)blockIdx.x ? c : 0;
+                total += c;
+            }
+        }
+        int32_t a = total;   // inclusive scan across the CTA
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t t = __shfl_up_sync(0xffffffffu, a, off);
+            if (lane >= off) a += t;
+        }
+        if (lane == 31) s_warp[warp] = a;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t wa = s_warp[lane];
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t t = __shfl_up_sync(0xffffffffu, wa, off);
+                if (lane >= off) wa += t;
+            }
+            s_warp[lane] = wa;
+        }
+        __syncthreads();
+        const int32_t base = s_carry + (warp ? s_warp[warp - 1] : 0);
+        if (j < k) {
+            const int32_t start = base + a - total;
+            s_next[j] = start + before;
+            if (blockIdx.x == 0) seg_start[j] = start;
+        }
+        __syncthreads();
+        if (tid == SORT_BLK - 1) s_carry = base + a;
+        __syncthreads();
+    }
+    if (blockIdx.x == 0 && tid == 0) seg_start[k] = s_carry;
+
     const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
     int32_t j = -1;
     if (i < b) {
@@ -194,6 +281,8 @@ contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, 
     __shared__ int32_t s_row[CT_TILE];
     __shared__ float s_alpha[CT_TILE];
     const int c = blockIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
     const int32_t total = seg_start[k];
     const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
     const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
@@ -286,6 +375,8 @@ contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_
                        float* __restrict__ Bt, int64_t ldb) {
     const int64_t mv = m_pad / 4;
     const int64_t idx = (int64_t)blockIdx.x * RED_THREADS + threadIdx.x;
+    grid_dependency_wait();
+    grid_launch_dependents();
     if (idx >= (int64_t)k * mv) return;
     const int j = (int)(idx / mv);
     const int64_t col = (idx % mv) * 4;

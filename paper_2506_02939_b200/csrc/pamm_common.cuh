@@ -17,6 +17,17 @@ __device__ int g_status_word;
 
 __device__ __forceinline__ void raise_status(int bit) { atomicOr(&g_status_word, bit); }
 
+// ---- programmatic dependent launch ---------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start
+// while its predecessor in the stream is still running.  It must call
+// grid_dependency_wait() before it touches anything the predecessor writes (or
+// anything the predecessor still reads and this kernel overwrites); the call
+// returns once the predecessor has finished and its writes are visible, and is
+// a no-op for an ordinary launch.  grid_launch_dependents() lets the successor's
+// CTAs be scheduled as soon as every CTA of this grid has issued it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- storage types ----------------------------------------------------------
 template <typename T> struct Vec16;   // 16 bytes of T
 template <> struct Vec16<float> {

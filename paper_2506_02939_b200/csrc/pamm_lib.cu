@@ -33,6 +33,25 @@ cudaEvent_t g_prof[3][2] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nu
 inline void prof_begin(int kind, cudaStream_t st) { if (g_prof[kind][0]) cudaEventRecord(g_prof[kind][0], st); }
 inline void prof_end(int kind, cudaStream_t st) { if (g_prof[kind][1]) cudaEventRecord(g_prof[kind][1], st); }
 
+// Launch with or without the programmatic-serialization attribute.  With it, the
+// kernel may begin while the previous kernel of the stream is still running and
+// must call grid_dependency_wait() before it depends on that kernel.
+template <typename... P, typename... A>
+inline void launch(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap_prev, A... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prev ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kern, P(args)...);
+    g_launches += 1;
+}
+
 struct StepArena {
     char *X, *dY, *C, *dW, *Bt, *ws;
     float *invnorm, *alpha;
@@ -75,9 +94,8 @@ pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int6
         return PAMM_ERR_CUDA;
     const PermKey pk = make_perm_key(seed, (uint32_t)b);
     const int grid = (int)((k + SEL_WARPS - 1) / SEL_WARPS);
-    select_kernel<T><<<grid, SEL_THREADS, smem, st>>>((const T*)X, ldx, b, n, (int)k, pk, idx_in, idx_out,
-                                                      (T*)C, ldc, c_invnorm);
-    g_launches += 1;
+    launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, false, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
+           idx_out, (T*)C, ldc, c_invnorm);
     return launch_status();
 }
 
@@ -88,15 +106,18 @@ pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t 
     const int grid = (int)std::min<int64_t>(want, 148 * 8);
     prof_begin(PAMM_PROF_COMPRESS, st);
     if (k <= 4)
-        compress_simt_kernel<T, 4><<<grid, CS_THREADS, 0, st>>>((const T*)X, ldx, b, n, (const T*)C, ldc, (int)k,
-                                                                c_invnorm, f, alpha);
+        launch(compress_simt_kernel<T, 4>, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C,
+               ldc, (int)k, c_invnorm, f, alpha);
     else
-        compress_simt_kernel<T, 8><<<grid, CS_THREADS, 0, st>>>((const T*)X, ldx, b, n, (const T*)C, ldc, (int)k,
-                                                                c_invnorm, f, alpha);
+        launch(compress_simt_kernel<T, 8>, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C,
+               ldc, (int)k, c_invnorm, f, alpha);
     prof_end(PAMM_PROF_COMPRESS, st);
-    g_launches += 1;
     return launch_status();
 }
+
+// Largest nb * nb * k (histogram words read by all scatter blocks together) for
+// which every block rebuilds the scan on its own instead of a separate launch.
+constexpr int64_t FUSED_SCAN_LIMIT = 1ll << 24;
 
 int sm_count() {
     static int sms = 0;
@@ -118,9 +139,15 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
         (cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess ||
          cudaFuncSetAttribute(contract_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess))
         return PAMM_ERR_CUDA;
-    contract_hist_kernel<<<(int)w.nb, SORT_BLK, hsmem, st>>>(f, b, (int)k, w.hist);
-    contract_scan_kernel<<<1, SCAN_THREADS, 0, st>>>(w.hist, (int)w.nb, (int)k, w.seg_start);
-    contract_scatter_kernel<<<(int)w.nb, SORT_BLK, hsmem, st>>>(f, b, (int)k, w.hist, w.seg_start, w.perm);
+    launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, false, f, b, (int)k, w.hist);
+    if (w.nb * w.nb * k <= FUSED_SCAN_LIMIT) {
+        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
+               (const int32_t*)w.hist, (int)w.nb, w.seg_start, w.perm);
+    } else {
+        launch(contract_scan_kernel, dim3(1), dim3(SCAN_THREADS), 0, st, true, w.hist, (int)w.nb, (int)k, w.seg_start);
+        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
+               (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
+    }
     // one balanced wave: every CTA gets the same number of sorted rows
     const int64_t vecs = (m + V - 1) / V;
     const int64_t slabs = (vecs + CT_MAX_THREADS - 1) / CT_MAX_THREADS;
@@ -133,13 +160,12 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
     ranges = (b + rows_per_cta - 1) / rows_per_cta;
     dim3 grid((unsigned)ranges, (unsigned)slabs);
     prof_begin(PAMM_PROF_CONTRACT, st);
-    contract_main_kernel<T><<<grid, threads, 0, st>>>(alpha, (const T*)dY, ldy, m, (int)k, w.seg_start, w.perm,
-                                                      (int)rows_per_cta, w.partials, w.m_pad, Bt, ldb);
+    launch(contract_main_kernel<T>, grid, dim3(threads), 0, st, true, alpha, (const T*)dY, ldy, m, (int)k,
+           (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, w.partials, w.m_pad, Bt, ldb);
     prof_end(PAMM_PROF_CONTRACT, st);
     const int64_t items = k * (w.m_pad / 4);
-    contract_reduce_kernel<<<(int)((items + RED_THREADS - 1) / RED_THREADS), RED_THREADS, 0, st>>>(
-        w.partials, w.m_pad, m, (int)k, w.seg_start, (int)rows_per_cta, Bt, ldb);
-    g_launches += 5;
+    launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st, true,
+           (const float*)w.partials, w.m_pad, m, (int)k, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
     return launch_status();
 }
 
@@ -148,10 +174,9 @@ pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64
                                     int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
     const int64_t items = n * ((m + 3) / 4);
     prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-    weight_grad_simt_kernel<T><<<(int)((items + WG_THREADS - 1) / WG_THREADS), WG_THREADS, 0, st>>>(
-        (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw);
+    launch(weight_grad_simt_kernel<T>, dim3((unsigned)((items + WG_THREADS - 1) / WG_THREADS)), dim3(WG_THREADS), 0, st, true,
+           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw);
     prof_end(PAMM_PROF_WEIGHT_GRAD, st);
-    g_launches += 1;
     return launch_status();
 }
 

@@ -2,7 +2,9 @@
 // and the norms of the generator rows).  One launch, no cross-CTA dependency:
 // every CTA recomputes the k candidate indices in shared memory, then each of
 // its warps ranks one candidate (rank = sorted position), copies that row of X
-// into C and accumulates its squared norm in fp64.
+// into C and accumulates its squared norm as an unevaluated fp32 pair (hi, lo)
+// with error-free additions, which carries about 48 bits: the stored 1/||C_j||
+// then has fp32 rounding only, at a fraction of the cost of fp64 arithmetic.
 #pragma once
 #include "pamm_common.cuh"
 
@@ -12,6 +14,15 @@ constexpr int SEL_THREADS = 256;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
 constexpr int64_t SEL_MAX_K = 49152;   // k * 4 bytes of dynamic shared memory
 
+// a <- fl(a + b); returns the rounding error of that addition (Knuth's branch-free form).
+__device__ __forceinline__ float two_sum(float& a, float b) {
+    const float s = __fadd_rn(a, b);
+    const float bb = __fsub_rn(s, a);
+    const float err = __fadd_rn(__fsub_rn(a, __fsub_rn(s, bb)), __fsub_rn(b, bb));
+    a = s;
+    return err;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(SEL_THREADS)
 select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k, PermKey pk,
@@ -19,6 +30,7 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
               T* __restrict__ C, int64_t ldc, float* __restrict__ c_invnorm) {
     extern __shared__ int32_t s_vals[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    grid_launch_dependents();   // the compress kernel may set itself up meanwhile
 
     for (int j = tid; j < k; j += SEL_THREADS)
         s_vals[j] = idx_in ? idx_in[j] : (int32_t)perm_apply(pk, (uint32_t)j);
@@ -54,7 +66,7 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
     constexpr int V = Vec16<T>::N;
     const T* src = X + (int64_t)val * ldx;
     T* dst = C + (int64_t)slot * ldc;
-    double q = 0.0;
+    float q_hi = 0.f, q_lo = 0.f;
     for (int64_t col = (int64_t)lane * V; col < n; col += 32 * V) {
         float x[V];
         load_vec<T>(src, col, n, x);
@@ -64,11 +76,20 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
             for (int e = 0; e < V && col + e < n; ++e) dst[col + e] = src[col + e];
         }
 #pragma unroll
-        for (int e = 0; e < V; ++e) q += (double)x[e] * (double)x[e];
+        for (int e = 0; e < V; ++e) {
+            const float p = __fmul_rn(x[e], x[e]);
+            const float pe = fmaf(x[e], x[e], -p);      // x^2 = p + pe exactly
+            q_lo += two_sum(q_hi, p) + pe;
+        }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) q += __shfl_xor_sync(0xffffffffu, q, off);
+    for (int off = 16; off > 0; off >>= 1) {   // the butterfly is symmetric: every lane ends with the same pair
+        const float o_hi = __shfl_xor_sync(0xffffffffu, q_hi, off);
+        const float o_lo = __shfl_xor_sync(0xffffffffu, q_lo, off);
+        q_lo = (q_lo + o_lo) + two_sum(q_hi, o_hi);
+    }
     if (lane == 0) {
+        const double q = (double)q_hi + (double)q_lo;
         idx_out[slot] = val;
         c_invnorm[slot] = (q > 0.0) ? (float)(1.0 / sqrt(q)) : 0.f;
         c_invnorm[k + slot] = (q > 0.0) ? (float)(1.0 / q) : 0.f;

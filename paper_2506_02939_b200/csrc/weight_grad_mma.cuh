@@ -68,6 +68,7 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
+    grid_dependency_wait();     // B~ (and C) may come from the kernel before
     // kind::f16, D fp32, A/B bf16, both MN-major (bits 15 and 16), M = N = 128
     const uint32_t idesc = ptx::umma_idesc_bf16(WU_TILE, WU_TILE) | (1u << 15) | (1u << 16);
     bool ok = true;
@@ -182,7 +183,17 @@ inline pamm_status launch_weight_grad_mma(const void* C, int64_t ldc, int64_t k,
     if (cudaFuncSetAttribute(weight_grad_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PAMM_ERR_CUDA;
     dim3 grid((unsigned)((m + WU_TILE - 1) / WU_TILE), (unsigned)((n + WU_TILE - 1) / WU_TILE));
-    weight_grad_umma_kernel<<<grid, WU_THREADS, smem, st>>>(tm_c, Bt, ldb, (int)k, (int)n, (int)m, kc, nchunks, dW, ldw);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(WU_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set up while the kernel before drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, weight_grad_umma_kernel, tm_c, Bt, ldb, (int)k, (int)n, (int)m, kc, nchunks, dW, ldw);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 
