@@ -169,29 +169,60 @@ contract_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const i
 // offset inside every segment (the counts of the blocks before it) -- and then
 // scatters its rows exactly as contract_scatter_kernel does.  Block 0 also
 // publishes seg_start.  Costs nb * k reads per block instead of a serial
-// single-CTA pass between two launches.
+// single-CTA pass between two launches.  The column sums are spread over all
+// threads: with W = the chunk's width rounded up to a power of two, the SORT_BLK
+// / W thread groups each take every (SORT_BLK / W)-th histogram row.
 __global__ void __launch_bounds__(SORT_BLK)
 contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const int32_t* __restrict__ hist,
                              int nb, int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
+    __shared__ int32_t s_part[2][SORT_BLK];   // per-thread partial (total, before) of the column sums
     __shared__ int32_t s_warp[32];
     __shared__ int32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int me = blockIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < k; j0 += SORT_BLK) {
-        const int j = j0 + tid;
+        const int width = min(SORT_BLK, k - j0);
+        int W = 32;
+        while (W < width) W <<= 1;
+        const int groups = SORT_BLK / W;
+        const int grp = tid / W, jj = tid % W;
         int32_t total = 0, before = 0;
-        if (j < k) {
-            for (int blk = 0; blk < nb; ++blk) {
-                const int32_t c = __ldg(hist + (int64_t)blk * k + j);
-                before += blk < (int)blockIdx.x ? c : 0;
+        if (jj < width) {
+            const int32_t* col = hist + j0 + jj;
+            int blk = grp;
+            for (; blk + 3 * groups < nb; blk += 4 * groups) {   // four independent loads in flight
+                const int32_t c0 = __ldg(col + (int64_t)blk * k);
+                const int32_t c1 = __ldg(col + (int64_t)(blk + groups) * k);
+                const int32_t c2 = __ldg(col + (int64_t)(blk + 2 * groups) * k);
+                const int32_t c3 = __ldg(col + (int64_t)(blk + 3 * groups) * k);
+                total += (c0 + c1) + (c2 + c3);
+                before += (blk < me ? c0 : 0) + (blk + groups < me ? c1 : 0) + (blk + 2 * groups < me ? c2 : 0) +
+                          (blk + 3 * groups < me ? c3 : 0);
+            }
+            for (; blk < nb; blk += groups) {
+                const int32_t c = __ldg(col + (int64_t)blk * k);
                 total += c;
+                before += blk < me ? c : 0;
             }
         }
-        int32_t a = total;   // inclusive scan across the CTA
+        s_part[0][tid] = total;
+        s_part[1][tid] = before;
+        __syncthreads();
+        total = 0;
+        before = 0;
+        if (tid < width) {
+            for (int g = 0; g < groups; ++g) {
+                total += s_part[0][g * W + tid];
+                before += s_part[1][g * W + tid];
+            }
+        }
+        const int j = j0 + tid;
+        int32_t a = total;   // inclusive scan across the CTA (threads beyond the chunk hold 0)
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const int32_t t = __shfl_up_sync(0xffffffffu, a, off);
@@ -210,16 +241,16 @@ contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, co
         }
         __syncthreads();
         const int32_t base = s_carry + (warp ? s_warp[warp - 1] : 0);
-        if (j < k) {
+        if (tid < width) {
             const int32_t start = base + a - total;
             s_next[j] = start + before;
-            if (blockIdx.x == 0) seg_start[j] = start;
+            if (me == 0) seg_start[j] = start;
         }
         __syncthreads();
         if (tid == SORT_BLK - 1) s_carry = base + a;
         __syncthreads();
     }
-    if (blockIdx.x == 0 && tid == 0) seg_start[k] = s_carry;
+    if (me == 0 && tid == 0) seg_start[k] = s_carry;
 
     const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
     int32_t j = -1;

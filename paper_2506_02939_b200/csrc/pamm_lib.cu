@@ -14,6 +14,7 @@
 #include "contract.cuh"
 #include "weight_grad_simt.cuh"
 #include "weight_grad_mma.cuh"
+#include "weight_grad_persist.cuh"
 
 using namespace pamm;
 
@@ -93,7 +94,7 @@ pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int6
         cudaFuncSetAttribute(select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PAMM_ERR_CUDA;
     const PermKey pk = make_perm_key(seed, (uint32_t)b);
-    const int grid = (int)((k + SEL_WARPS - 1) / SEL_WARPS);
+    const int grid = (int)k;
     launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, false, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
            idx_out, (T*)C, ldc, c_invnorm);
     return launch_status();
@@ -242,6 +243,13 @@ pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_d
 pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
                            int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
     if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+    if (weight_grad_persist_supported(k, n, m)) {
+        prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
+        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st);
+        prof_end(PAMM_PROF_WEIGHT_GRAD, st);
+        g_launches += 1;
+        return s;
+    }
     if (weight_grad_mma_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
         const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);

@@ -1,8 +1,8 @@
 // Step 1: generator selection (Algorithm 1: "Sample indices I", "C <- A[I,:]",
 // and the norms of the generator rows).  One launch, no cross-CTA dependency:
-// every CTA recomputes the k candidate indices in shared memory, then each of
-// its warps ranks one candidate (rank = sorted position), copies that row of X
-// into C and accumulates its squared norm as an unevaluated fp32 pair (hi, lo)
+// every CTA recomputes the k candidate indices in shared memory, ranks its own
+// candidate (rank = sorted position), copies that row of X into C with one
+// 16-byte load per thread and accumulates its squared norm as an unevaluated fp32 pair (hi, lo)
 // with error-free additions, which carries about 48 bits: the stored 1/||C_j||
 // then has fp32 rounding only, at a fraction of the cost of fp64 arithmetic.
 #pragma once
@@ -29,6 +29,8 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
               const int32_t* __restrict__ idx_in, int32_t* __restrict__ idx_out,
               T* __restrict__ C, int64_t ldc, float* __restrict__ c_invnorm) {
     extern __shared__ int32_t s_vals[];
+    __shared__ int s_cnt[2][SEL_WARPS];
+    __shared__ float s_q[2][SEL_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     grid_launch_dependents();   // the compress kernel may set itself up meanwhile
 
@@ -36,14 +38,13 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
         s_vals[j] = idx_in ? idx_in[j] : (int32_t)perm_apply(pk, (uint32_t)j);
     __syncthreads();
 
-    const int j = blockIdx.x * SEL_WARPS + warp;
-    if (j >= k) return;
+    const int j = blockIdx.x;          // one CTA per generator
     int32_t val = s_vals[j];
 
-    // rank among all candidates, and a duplicate count (warp-wide)
+    // rank among all candidates, and a duplicate count
     int smaller = 0, dup = 0;
-    for (int t = lane; t < k; t += 32) {
-        int32_t o = s_vals[t];
+    for (int t = tid; t < k; t += SEL_THREADS) {
+        const int32_t o = s_vals[t];
         smaller += (o < val);
         dup += (o == val && t != j);
     }
@@ -52,13 +53,20 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
         smaller += __shfl_xor_sync(0xffffffffu, smaller, off);
         dup += __shfl_xor_sync(0xffffffffu, dup, off);
     }
+    if (lane == 0) { s_cnt[0][warp] = smaller; s_cnt[1][warp] = dup; }
+    __syncthreads();
+    smaller = 0;
+    dup = 0;
+#pragma unroll
+    for (int w = 0; w < SEL_WARPS; ++w) { smaller += s_cnt[0][w]; dup += s_cnt[1][w]; }
+
     int slot;
     if (idx_in) {
         slot = j;   // caller's order
         bool bad = dup > 0;
         if (val < 0) { val = 0; bad = true; }
         if ((int64_t)val >= b) { val = (int32_t)(b - 1); bad = true; }
-        if (bad && lane == 0) raise_status(DEV_BAD_INDEX);
+        if (bad && tid == 0) raise_status(DEV_BAD_INDEX);
     } else {
         slot = smaller;   // distinct by construction: rank = ascending position
     }
@@ -67,7 +75,7 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
     const T* src = X + (int64_t)val * ldx;
     T* dst = C + (int64_t)slot * ldc;
     float q_hi = 0.f, q_lo = 0.f;
-    for (int64_t col = (int64_t)lane * V; col < n; col += 32 * V) {
+    for (int64_t col = (int64_t)tid * V; col < n; col += SEL_THREADS * V) {
         float x[V];
         load_vec<T>(src, col, n, x);
         if (col + V <= n) {
@@ -83,13 +91,17 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
         }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {   // the butterfly is symmetric: every lane ends with the same pair
+    for (int off = 16; off > 0; off >>= 1) {
         const float o_hi = __shfl_xor_sync(0xffffffffu, q_hi, off);
         const float o_lo = __shfl_xor_sync(0xffffffffu, q_lo, off);
         q_lo = (q_lo + o_lo) + two_sum(q_hi, o_hi);
     }
-    if (lane == 0) {
-        const double q = (double)q_hi + (double)q_lo;
+    if (lane == 0) { s_q[0][warp] = q_hi; s_q[1][warp] = q_lo; }
+    __syncthreads();
+    if (tid == 0) {
+        double q = 0.0;     // eight pairs, added in warp order
+#pragma unroll
+        for (int w = 0; w < SEL_WARPS; ++w) q += (double)s_q[0][w] + (double)s_q[1][w];
         idx_out[slot] = val;
         c_invnorm[slot] = (q > 0.0) ? (float)(1.0 / sqrt(q)) : 0.f;
         c_invnorm[k + slot] = (q > 0.0) ? (float)(1.0 / q) : 0.f;
