@@ -24,7 +24,10 @@ namespace pamm {
 constexpr int CU_THREADS = 192;
 constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
 constexpr int CU_TILE_M = 128;
-constexpr int CU_BOX_ROWS = 32;
+#ifndef PAMM_CU_BOX_ROWS
+#define PAMM_CU_BOX_ROWS 32
+#endif
+constexpr int CU_BOX_ROWS = PAMM_CU_BOX_ROWS;
 constexpr int CU_X_TILE_BYTES = CU_TILE_M * 128;   // 16 KiB
 constexpr int CU_MAX_K = 4096;                 // 1/||C_j|| and 1/||C_j||^2 live in shared memory
 constexpr int CU_SMEM_BUDGET = 200 * 1024;

@@ -12,6 +12,7 @@
 #include "compress_simt.cuh"
 #include "compress_umma.cuh"
 #include "contract.cuh"
+#include "contract_stream.cuh"
 #include "weight_grad_simt.cuh"
 #include "weight_grad_mma.cuh"
 #include "weight_grad_persist.cuh"
@@ -149,7 +150,27 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
         launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
                (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
     }
-    // one balanced wave: every CTA gets the same number of sorted rows
+    if (contract_stream_supported(m, sizeof(T))) {
+        // one balanced wave, one CTA per SM: rows of dY stream through a shared-memory ring
+        const ContractStreamPlan p = contract_stream_plan(m, sizeof(T));
+        int64_t ranges = std::min<int64_t>(CT_MAX_CTAS, (int64_t)sm_count() * CS_CTAS_PER_SM);
+        const int64_t rows_per_cta = std::max<int64_t>(32, (b + ranges - 1) / ranges);
+        ranges = (b + rows_per_cta - 1) / rows_per_cta;
+        auto kern = p.vpt == 1 ? contract_stream_kernel<T, 1> : p.vpt == 2 ? contract_stream_kernel<T, 2>
+                                                                           : contract_stream_kernel<T, 4>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
+            return PAMM_ERR_CUDA;
+        prof_begin(PAMM_PROF_CONTRACT, st);
+        launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, alpha, (const T*)dY, ldy, m,
+               (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots, p.slot_bytes,
+               p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
+        prof_end(PAMM_PROF_CONTRACT, st);
+        const int64_t items = k * (w.m_pad / 4);
+        launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st,
+               true, (const float*)w.partials, w.m_pad, m, (int)k, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
+        return launch_status();
+    }
+    // very wide rows: column slabs, register staging
     const int64_t vecs = (m + V - 1) / V;
     const int64_t slabs = (vecs + CT_MAX_THREADS - 1) / CT_MAX_THREADS;
     const int threads = (int)round_up((vecs + slabs - 1) / slabs, 32);

@@ -28,6 +28,9 @@ SMALL = [
     (640, 64, 6152, 96, "bf16"),
     (129, 8, 8, 129, "bf16"),
     (5000, 1024, 256, 256, "bf16"),
+    (260, 24, 12280, 8, "bf16"),       # dY rows of 24 KiB: four 16-byte chunks per consumer thread
+    (96, 16, 24584, 8, "bf16"),        # rows too wide for the shared-memory ring: column-slab path
+    (333, 40, 3076, 6, "f32"),         # fp32 rows of 769 chunks: two per consumer thread
 ]
 
 
