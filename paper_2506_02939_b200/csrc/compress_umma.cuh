@@ -25,7 +25,7 @@ constexpr int CU_THREADS = 192;
 constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
 constexpr int CU_TILE_M = 128;
 #ifndef PAMM_CU_BOX_ROWS
-#define PAMM_CU_BOX_ROWS 32
+#define PAMM_CU_BOX_ROWS 64
 #endif
 constexpr int CU_BOX_ROWS = PAMM_CU_BOX_ROWS;
 constexpr int CU_X_TILE_BYTES = CU_TILE_M * 128;   // 16 KiB
@@ -110,6 +110,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_x);
             ptx::prefetch_tensormap(&tm_c);
+            const uint64_t stream_policy = ptx::l2_policy_evict_first();   // X is read once; C stays in L2
             uint32_t it = 0;
             bool ok = true;
             for (int64_t st = r0; st < r1 && ok; st += super_rows) {
@@ -131,9 +132,9 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
                         for (int mt = 0; mt < MT; ++mt)
                             for (int q = 0; q < boxes[mt]; ++q)
-                                ptx::tma_load_2d(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
-                                                 ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
-                                                 &s_full[s]);
+                                ptx::tma_load_2d_hint(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
+                                                      ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
+                                                      &s_full[s], stream_policy);
                         ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, ch * n_chunk, &s_full[s]);
                     }
                 }

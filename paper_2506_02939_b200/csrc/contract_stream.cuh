@@ -121,6 +121,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
             j_cur = f[i_cur];
         }
         if (r + slots < r_end) i_nxt = perm[r + slots];
+        const uint64_t stream_policy = ptx::l2_policy_evict_first();   // dY is read once
         uint32_t phase = 0, idle = 0;
         bool issued = false, ok = true;
         uint32_t issued_phase = 0;
@@ -130,7 +131,8 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                 s_meta[lane] = make_int4(i_cur, j_cur, __float_as_int(a_cur), 0);
                 if (bulk_bytes) {
                     ptx::mbar_arrive_expect_tx(&s_full[lane], bulk_bytes);
-                    ptx::bulk_load(ring + (size_t)lane * slot_bytes, dY + (int64_t)i_cur * ldy, bulk_bytes, &s_full[lane]);
+                    ptx::bulk_load_hint(ring + (size_t)lane * slot_bytes, dY + (int64_t)i_cur * ldy, bulk_bytes, &s_full[lane],
+                                        stream_policy);
                 } else {
                     ptx::mbar_arrive(&s_full[lane]);
                 }
