@@ -23,6 +23,7 @@ compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
     const int64_t warp0 = (int64_t)blockIdx.x * CS_WARPS + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * CS_WARPS;
     grid_dependency_wait();     // C and the norms come from the kernel before
+    grid_launch_dependents();
 
     for (int64_t i = warp0; i < b; i += nwarps) {
         const T* xrow = X + i * ldx;

@@ -70,7 +70,7 @@ template <int MT>
 __global__ void __launch_bounds__(CU_THREADS, 1)
 compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
                      int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
-                     int tmem_cols, int rows_per_cta, const float* __restrict__ c_invnorm,
+                     int tmem_cols, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
                      int32_t* __restrict__ f, float* __restrict__ alpha) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2];
@@ -97,8 +97,11 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         ptx::tmem_alloc(&s_tmem_base, (uint32_t)tmem_cols);
         ptx::tmem_relinquish();
     }
-    grid_dependency_wait();     // C and the norms come from the kernel before
-    for (int j = threadIdx.x; j < 2 * k; j += CU_THREADS) s_inv[j] = c_invnorm[j];
+    grid_launch_dependents();   // the next kernel of the stream may set itself up meanwhile
+    // C and the norms come from the kernel before.  When the caller vouches that X was
+    // complete before that kernel started, the producer streams the first X tiles while
+    // it still runs and everybody else waits for it only where C or the norms are read.
+    if (!x_is_ready) grid_dependency_wait();
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -111,33 +114,46 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             ptx::prefetch_tensormap(&tm_x);
             ptx::prefetch_tensormap(&tm_c);
             const uint64_t stream_policy = ptx::l2_policy_evict_first();   // X is read once; C stays in L2
+            // pipeline step `it` = (row super tile, generator chunk, 64-column step), flattened
+            const uint32_t per_super = (uint32_t)(num_chunks * ksteps);
+            const uint32_t total = (uint32_t)((r1 - r0 + super_rows - 1) / super_rows) * per_super;
+            auto issue = [&](uint32_t at, bool with_x, bool with_c, bool arm) {
+                const int64_t st = r0 + (int64_t)(at / per_super) * super_rows;
+                const int ch = (int)((at % per_super) / (uint32_t)ksteps), ks = (int)(at % (uint32_t)ksteps);
+                const int s = at % stages;
+                uint8_t* stage = tiles + (size_t)s * stage_bytes;
+                uint32_t bytes = (uint32_t)n_chunk * 128u;
+                int boxes[MT];
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const int64_t rows = min((int64_t)CU_TILE_M, r1 - (st + (int64_t)mt * CU_TILE_M));
+                    boxes[mt] = rows > 0 ? (int)((rows + CU_BOX_ROWS - 1) / CU_BOX_ROWS) : 0;
+                    bytes += (uint32_t)boxes[mt] * (CU_BOX_ROWS * 128u);
+                }
+                if (arm) ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
+                if (with_x) {
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+                        for (int q = 0; q < boxes[mt]; ++q)
+                            ptx::tma_load_2d_hint(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
+                                                  ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
+                                                  &s_full[s], stream_policy);
+                }
+                if (with_c)
+                    ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, ch * n_chunk, &s_full[s]);
+            };
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t st = r0; st < r1 && ok; st += super_rows) {
-                for (int ch = 0; ch < num_chunks && ok; ++ch) {
-                    for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                        const int s = it % stages;
-                        const uint32_t ph = (it / stages) & 1u;
-                        if (!ptx::mbar_wait(&s_empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-                        uint8_t* stage = tiles + (size_t)s * stage_bytes;
-                        uint32_t bytes = (uint32_t)n_chunk * 128u;
-                        int boxes[MT];
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt) {
-                            const int64_t rows = min((int64_t)CU_TILE_M, r1 - (st + (int64_t)mt * CU_TILE_M));
-                            boxes[mt] = rows > 0 ? (int)((rows + CU_BOX_ROWS - 1) / CU_BOX_ROWS) : 0;
-                            bytes += (uint32_t)boxes[mt] * (CU_BOX_ROWS * 128u);
-                        }
-                        ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt)
-                            for (int q = 0; q < boxes[mt]; ++q)
-                                ptx::tma_load_2d_hint(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
-                                                      ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
-                                                      &s_full[s], stream_policy);
-                        ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, ch * n_chunk, &s_full[s]);
-                    }
-                }
+            if (x_is_ready) {     // fill the ring with X, then wait for the kernel before, then add the C tiles
+                const uint32_t ahead = total < (uint32_t)stages ? total : (uint32_t)stages;
+                for (uint32_t a = 0; a < ahead; ++a) issue(a, true, false, true);
+                grid_dependency_wait();
+                for (uint32_t a = 0; a < ahead; ++a) issue(a, false, true, false);
+                it = ahead;
+            }
+            for (; it < total; ++it) {
+                if (!ptx::mbar_wait(&s_empty[it % stages], ((it / stages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                issue(it, true, true, true);
             }
             if (!ok) {
                 raise_status(DEV_TIMEOUT);
@@ -189,6 +205,9 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         // ---------------- epilogue: one row per thread ----------------
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
         const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
+        if (x_is_ready) grid_dependency_wait();
+        for (int j = threadIdx.x - 64; j < 2 * k; j += 128) s_inv[j] = c_invnorm[j];
+        ptx::named_barrier(1, 128);                      // the four epilogue warps share s_inv
         uint32_t unit = 0;
         bool ok = true;
         for (int64_t st = r0; st < r1 && ok; st += super_rows) {
@@ -249,7 +268,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 
 inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
                                         int64_t k, const float* c_invnorm, int32_t* f, float* alpha, int sms,
-                                        cudaStream_t st) {
+                                        bool x_is_ready, cudaStream_t st) {
     const CompressUmmaPlan p = compress_umma_plan(b, k, sms);
     CUtensorMap tm_x, tm_c;
     if (!make_tmap_bf16_sw128(&tm_x, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, CU_BOX_ROWS) ||
@@ -269,7 +288,7 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
-                       p.tmem_cols, p.rows_per_cta, c_invnorm, f, alpha);
+                       p.tmem_cols, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

@@ -61,8 +61,9 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
 __global__ void __launch_bounds__(SORT_BLK)
 contract_hist_kernel(const int32_t* __restrict__ f, int64_t b, int k, int32_t* __restrict__ hist) {
     extern __shared__ int32_t s_hist[];
-    grid_launch_dependents();
     for (int j = threadIdx.x; j < k; j += SORT_BLK) s_hist[j] = 0;
+    grid_dependency_wait();     // f may come from the kernel before
+    grid_launch_dependents();
     __syncthreads();
     const int64_t i = (int64_t)blockIdx.x * SORT_BLK + threadIdx.x;
     if (i < b) {

@@ -96,7 +96,7 @@ pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int6
         return PAMM_ERR_CUDA;
     const PermKey pk = make_perm_key(seed, (uint32_t)b);
     const int grid = (int)k;
-    launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, false, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
+    launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, true, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
            idx_out, (T*)C, ldc, c_invnorm);
     return launch_status();
 }
@@ -141,7 +141,7 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
         (cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess ||
          cudaFuncSetAttribute(contract_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess))
         return PAMM_ERR_CUDA;
-    launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, false, f, b, (int)k, w.hist);
+    launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k, w.hist);
     if (w.nb * w.nb * k <= FUSED_SCAN_LIMIT) {
         launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
                (const int32_t*)w.hist, (int)w.nb, w.seg_start, w.perm);
@@ -248,12 +248,15 @@ pamm_status check_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, 
     return PAMM_OK;
 }
 
+// x_is_ready: X was complete before the previous kernel of the stream started (true
+// after our own select kernel), so the compress kernel may read it before that
+// kernel has finished.
 pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
-                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, cudaStream_t st) {
+                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, bool x_is_ready, cudaStream_t st) {
     if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
     if (compress_umma_supported(b, n, k)) {
         prof_begin(PAMM_PROF_COMPRESS, st);
-        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), st);
+        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), x_is_ready, st);
         prof_end(PAMM_PROF_COMPRESS, st);
         g_launches += 1;
         return s;
@@ -349,7 +352,7 @@ pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm
     (void)workspace; (void)ws_bytes;
     pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
     if (s != PAMM_OK) return s;
-    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, (cudaStream_t)stream);
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, false, (cudaStream_t)stream);
 }
 
 pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, int64_t k,
@@ -365,7 +368,7 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
     s = dt == PAMM_F32 ? launch_select<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st)
                        : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
     if (s != PAMM_OK) return s;
-    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, st);
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, true, st);
 }
 
 pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,

@@ -32,10 +32,15 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
     __shared__ int s_cnt[2][SEL_WARPS];
     __shared__ float s_q[2][SEL_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    grid_launch_dependents();   // the compress kernel may set itself up meanwhile
-
-    for (int j = tid; j < k; j += SEL_THREADS)
-        s_vals[j] = idx_in ? idx_in[j] : (int32_t)perm_apply(pk, (uint32_t)j);
+    // Drawn indices need no memory, so they are computed while the kernel before may
+    // still be running; everything read from memory comes after the wait.  Only then
+    // is the compress kernel let in: it may read X as soon as it starts.
+    if (!idx_in)
+        for (int j = tid; j < k; j += SEL_THREADS) s_vals[j] = (int32_t)perm_apply(pk, (uint32_t)j);
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if (idx_in)
+        for (int j = tid; j < k; j += SEL_THREADS) s_vals[j] = idx_in[j];
     __syncthreads();
 
     const int j = blockIdx.x;          // one CTA per generator

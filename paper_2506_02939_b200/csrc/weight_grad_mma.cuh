@@ -69,6 +69,7 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
     grid_dependency_wait();     // B~ (and C) may come from the kernel before
+    grid_launch_dependents();
     // kind::f16, D fp32, A/B bf16, both MN-major (bits 15 and 16), M = N = 128
     const uint32_t idesc = ptx::umma_idesc_bf16(WU_TILE, WU_TILE) | (1u << 15) | (1u << 16);
     bool ok = true;

@@ -88,6 +88,7 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
     grid_dependency_wait();     // B~ (and C) may come from the kernel before
+    grid_launch_dependents();
 
     if (warp == 0) {
         // ---------------- TMA producer: C tiles ----------------

@@ -24,6 +24,7 @@ weight_grad_simt_kernel(const T* __restrict__ C, int64_t ldc, int k, int64_t n,
     const int64_t mv = (m + 3) / 4;
     const int64_t idx = (int64_t)blockIdx.x * WG_THREADS + threadIdx.x;
     grid_dependency_wait();     // B~ (and C) may come from the kernel before
+    grid_launch_dependents();
     if (idx >= n * mv) return;
     const int64_t r = idx / mv, col = (idx % mv) * 4;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
