@@ -33,7 +33,7 @@ PROF_EVERY = 16     # one step in PROF_EVERY carries per-kernel CUDA events, ano
                     # the rest run event-free, since an event between two kernels serialises their launches
 # DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
 # summarised under profiles/, keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"c4": 812307456}     # contract_stream_kernel<bf16,2>: 806.12 MB read + 6.19 MB written
 
 
 def env_int(name, default):
@@ -354,7 +354,7 @@ def run_cuda(args):
                    "l2": "inputs exceed L2 (X %.0f MiB, dY %.0f MiB per step)" % (b * n * e / 2**20, b * m * e / 2**20)
                    if b * n * e > 126 * 2**20 else "inputs fit L2: warm-cache numbers",
                    "parallelism": f"replicas x{world}"},
-        "roofline": {"bound": "hbm", "kernel": "contract_main", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "contract_stream_kernel (contract main pass)", "achieved": achieved, "peak": peak,
                      "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(w.name), "algorithmic_bytes": ab["contract"]},
         "cpu_baseline": cpu,
