@@ -62,8 +62,39 @@ inline CompressUmmaPlan compress_umma_plan(int64_t b, int64_t k, int sms) {
     const int64_t per = (b + sms - 1) / sms;
     p.rows_per_cta = (int)std::max<int64_t>(CU_BOX_ROWS, round_up(per, CU_BOX_ROWS));
     p.grid = (int)((b + p.rows_per_cta - 1) / p.rows_per_cta);
-    p.smem_bytes = 1024 + (size_t)p.stages * p.stage_bytes + (size_t)2 * k * 4 + 256;
+    p.smem_bytes = 1024 + (size_t)p.stages * p.stage_bytes + (size_t)(p.num_chunks * p.n_chunk + k) * 4 + 256;
     return p;
+}
+
+// Folds 16 consecutive scores |s_i| * inv_i into the running (best score, its dot
+// product, its index).  A left-biased tournament: at every node the right entry
+// wins only if strictly larger, so the lowest index keeps a tie, exactly as an
+// ascending scan with '>' would -- but four levels deep instead of sixteen.
+__device__ __forceinline__ void argmax16(const uint32_t (&v)[16], const float* __restrict__ inv, int j0,
+                                         float& best, float& s_best, int& j_best) {
+    float sc[16], sv[16];
+    int ji[16];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 w = *reinterpret_cast<const float4*>(inv + 4 * q);
+        sv[4 * q] = __uint_as_float(v[4 * q]);         sc[4 * q] = fabsf(sv[4 * q]) * w.x;
+        sv[4 * q + 1] = __uint_as_float(v[4 * q + 1]); sc[4 * q + 1] = fabsf(sv[4 * q + 1]) * w.y;
+        sv[4 * q + 2] = __uint_as_float(v[4 * q + 2]); sc[4 * q + 2] = fabsf(sv[4 * q + 2]) * w.z;
+        sv[4 * q + 3] = __uint_as_float(v[4 * q + 3]); sc[4 * q + 3] = fabsf(sv[4 * q + 3]) * w.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) ji[i] = i;
+#pragma unroll
+    for (int width = 1; width < 16; width <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 16; i += 2 * width) {
+            const bool right = sc[i + width] > sc[i];
+            sc[i] = right ? sc[i + width] : sc[i];
+            sv[i] = right ? sv[i + width] : sv[i];
+            ji[i] = right ? ji[i + width] : ji[i];
+        }
+    }
+    if (sc[0] > best) { best = sc[0]; s_best = sv[0]; j_best = j0 + ji[0]; }
 }
 
 template <int MT>
@@ -79,7 +110,11 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    float* s_inv = reinterpret_cast<float*>(tiles + (size_t)stages * stage_bytes);   // [0,k) 1/||C||, [k,2k) 1/||C||^2
+    // 1/||C_j|| for every column the chunks cover, zero beyond k (a padded column scores 0
+    // and never beats a real one), then 1/||C_j||^2
+    const int kpad = n_chunk * num_chunks;
+    float* s_inv = reinterpret_cast<float*>(tiles + (size_t)stages * stage_bytes);
+    float* s_inv2 = s_inv + kpad;
 
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
     const int64_t r1 = min(b, r0 + (int64_t)rows_per_cta);
@@ -206,8 +241,9 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
         const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
         if (x_is_ready) grid_dependency_wait();
-        for (int j = threadIdx.x - 64; j < 2 * k; j += 128) s_inv[j] = c_invnorm[j];
-        ptx::named_barrier(1, 128);                      // the four epilogue warps share s_inv
+        for (int j = threadIdx.x - 64; j < kpad; j += 128) s_inv[j] = j < k ? c_invnorm[j] : 0.f;
+        for (int j = threadIdx.x - 64; j < k; j += 128) s_inv2[j] = c_invnorm[k + j];
+        ptx::named_barrier(1, 128);                      // the four epilogue warps share the norms
         uint32_t unit = 0;
         bool ok = true;
         for (int64_t st = r0; st < r1 && ok; st += super_rows) {
@@ -224,19 +260,21 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     if (st + (int64_t)mt * CU_TILE_M >= r1) continue;
-                    for (int c0 = 0; c0 < n_chunk; c0 += 16) {
-                        uint32_t v[16];
-                        ptx::tmem_ld_16cols(d_base + (uint32_t)(mt * n_chunk + c0), v);
-                        ptx::tmem_ld_wait();
-                        const int jb = ch * n_chunk + c0;
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int j = jb + i;
-                            if (j < k) {
-                                const float s = __uint_as_float(v[i]);
-                                const float score = fabsf(s) * s_inv[j];
-                                if (score > best[mt]) { best[mt] = score; s_best[mt] = s; j_best[mt] = j; }
-                            }
+                    // two register buffers: the TMEM load of the next 16 columns is in flight
+                    // while the current 16 go through the tournament
+                    const uint32_t t_base = d_base + (uint32_t)(mt * n_chunk);
+                    const int jb = ch * n_chunk;
+                    uint32_t va[16], vb[16];
+                    ptx::tmem_ld_16cols(t_base, va);
+                    for (int c0 = 0; c0 < n_chunk; c0 += 32) {
+                        ptx::tmem_ld_wait(va);
+                        const bool second = c0 + 16 < n_chunk;
+                        if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
+                        argmax16(va, s_inv + jb + c0, jb + c0, best[mt], s_best[mt], j_best[mt]);
+                        if (second) {
+                            ptx::tmem_ld_wait(vb);
+                            if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
+                            argmax16(vb, s_inv + jb + c0 + 16, jb + c0 + 16, best[mt], s_best[mt], j_best[mt]);
                         }
                     }
                 }
@@ -250,7 +288,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                     const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
                     if (row < r1) {
                         f[row] = j_best[mt];
-                        alpha[row] = s_best[mt] * s_inv[k + j_best[mt]];
+                        alpha[row] = s_best[mt] * s_inv2[j_best[mt]];
                     }
                 }
             }
