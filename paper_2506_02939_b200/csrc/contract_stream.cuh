@@ -6,7 +6,9 @@
 // CTAs per SM in a single balanced wave (two independent pipelines per SM hide
 // each other's waits; measured 17% faster than one CTA with twice the ring).
 // Inside a CTA:
-//   warp 0      producer: lane l owns ring slot l.  A round of the ring is handled by
+//   warp 0      producer: lane l owns ring slot l (a slot holds R = 1, 2 or 4 rows, so that
+//               a slot is 8-16 KB whatever the row width and the per-slot handshake is
+//               amortised over narrow rows).  A round of the ring is handled by
 //               all lanes at once: each looks its row up (perm -> row id, alpha, f; one
 //               round ahead), waits for its slot to be free and issues one
 //               cp.async.bulk for the row, so the whole ring (88 KB per CTA) is in
@@ -36,16 +38,26 @@ namespace pamm {
 #endif
 constexpr int CS_CTAS_PER_SM = PAMM_CS_CTAS_PER_SM;       // the ring budget is per CTA
 constexpr int CS_MAX_CONSUMERS = PAMM_CS_MAX_CONSUMERS;   // consumer threads
+#ifndef PAMM_CS_MIN_VPT
+#define PAMM_CS_MIN_VPT 1
+#endif
+constexpr int CS_MIN_VPT = PAMM_CS_MIN_VPT;
 constexpr int CS_MAX_VPT = 4;                    // 16-byte chunks per consumer thread
 constexpr int CS_MAX_SLOTS = 32;
+#ifndef PAMM_CS_MAX_RPS
+#define PAMM_CS_MAX_RPS 4
+#endif
+constexpr int CS_MAX_RPS = PAMM_CS_MAX_RPS;      // rows per ring slot, at most
+constexpr int CS_SLOT_TARGET_BYTES = 16 * 1024;  // rows are grouped while the slot stays within this
 constexpr uint32_t CS_PRODUCER_SPINS = 1u << 22;  // idle polls before the producer gives up
 constexpr int CS_RING_BYTES = PAMM_CS_RING_KB * 1024;
 
 struct ContractStreamPlan {
     int consumers;      // consumer threads, a multiple of 32
     int vpt;            // chunks per consumer thread (1, 2 or 4)
+    int rps;            // rows per ring slot (1, 2 or 4; more than 1 only with vpt == 1)
     int slots;
-    int slot_bytes;
+    int row_pitch;      // bytes between the rows of a slot
     uint32_t bulk_bytes;   // bytes of a row copied by the bulk engine (a multiple of 16)
     size_t smem_bytes;
 };
@@ -60,31 +72,35 @@ inline ContractStreamPlan contract_stream_plan(int64_t m, size_t esz) {
     ContractStreamPlan p;
     const int64_t row_bytes = m * (int64_t)esz;
     const int64_t vecs = (row_bytes + 15) / 16;
-    p.vpt = 1;
+    p.vpt = CS_MIN_VPT;
     while ((vecs + p.vpt - 1) / p.vpt > CS_MAX_CONSUMERS) p.vpt *= 2;
     p.consumers = (int)round_up((vecs + p.vpt - 1) / p.vpt, 32);
     p.bulk_bytes = (uint32_t)(row_bytes & ~(int64_t)15);
-    p.slot_bytes = (int)round_up(std::max<int64_t>(p.bulk_bytes, 16), 128);
-    p.slots = std::max(2, std::min(CS_MAX_SLOTS, CS_RING_BYTES / p.slot_bytes));
-    p.smem_bytes = 128 + (size_t)p.slots * p.slot_bytes;
+    p.row_pitch = (int)round_up(std::max<int64_t>(p.bulk_bytes, 16), 128);
+    p.rps = 1;
+    if (p.vpt == 1)
+        while (p.rps < CS_MAX_RPS && 2 * p.rps * p.row_pitch <= CS_SLOT_TARGET_BYTES) p.rps *= 2;
+    p.slots = std::max(2, std::min(CS_MAX_SLOTS, CS_RING_BYTES / (p.rps * p.row_pitch)));
+    p.smem_bytes = 128 + (size_t)p.slots * p.rps * p.row_pitch;
     return p;
 }
 
-template <typename T, int VPT>
+template <typename T, int VPT, int RPS>
 __global__ void __launch_bounds__(CS_MAX_CONSUMERS + 32, CS_CTAS_PER_SM)
 contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ alpha, const T* __restrict__ dY,
                        int64_t ldy, int64_t m, int k, const int32_t* __restrict__ seg_start,
-                       const int32_t* __restrict__ perm, int rows_per_cta, int slots, int slot_bytes,
+                       const int32_t* __restrict__ perm, int rows_per_cta, int slots, int row_pitch,
                        uint32_t bulk_bytes, float* __restrict__ partials, int64_t m_pad,
                        float* __restrict__ Bt, int64_t ldb) {
     constexpr int V = Vec16<T>::N;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[CS_MAX_SLOTS], s_empty[CS_MAX_SLOTS];
-    __shared__ int4 s_meta[CS_MAX_SLOTS];      // row id, generator, alpha bits of the row in the slot
+    __shared__ int4 s_meta[CS_MAX_SLOTS][RPS];      // row id, generator, alpha bits of every row in the slot
     __shared__ int s_abort;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int consumers = blockDim.x - 32;
     uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const int slot_bytes = RPS * row_pitch;
     const int c = blockIdx.x;
 
     if (tid == 0) {
@@ -108,19 +124,25 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
 
     if (warp == 0) {
         // ---------------- producer ----------------
-        // Lane l owns slot l and the rows r_begin + l, + slots, + 2 slots, ...  Every
-        // lane refills its slot as soon as the consumers hand it back, independently of
-        // the other lanes (a non-blocking test per poll).  Look-ups run ahead: the row
-        // id two rounds ahead, alpha and f one round ahead, so no poll waits on them.
-        int32_t r = lane < slots ? r_begin + lane : r_end;     // my next row (sorted position)
-        int32_t i_cur = -1, i_nxt = -1, j_cur = 0;
-        float a_cur = 0.f;
-        if (r < r_end) {
-            i_cur = perm[r];
-            a_cur = alpha[i_cur];
-            j_cur = f[i_cur];
+        // Lane l owns slot l and, in every round of the ring, the RPS consecutive sorted
+        // rows that go into it.  Every lane refills its slot as soon as the consumers hand
+        // it back, independently of the other lanes (a non-blocking test per poll).
+        // Look-ups run ahead: the row ids two rounds ahead, alpha and f one round ahead,
+        // so no poll waits on them.
+        const int32_t round_rows = slots * RPS;
+        int32_t r = lane < slots ? r_begin + lane * RPS : r_end;     // first sorted position of my next slot load
+        int32_t i_cur[RPS], i_nxt[RPS], j_cur[RPS];
+        float a_cur[RPS];
+#pragma unroll
+        for (int u = 0; u < RPS; ++u) {
+            i_cur[u] = -1; i_nxt[u] = -1; j_cur[u] = 0; a_cur[u] = 0.f;
+            if (r + u < r_end) {
+                i_cur[u] = perm[r + u];
+                a_cur[u] = alpha[i_cur[u]];
+                j_cur[u] = f[i_cur[u]];
+            }
+            if (r + round_rows + u < r_end) i_nxt[u] = perm[r + round_rows + u];
         }
-        if (r + slots < r_end) i_nxt = perm[r + slots];
         const uint64_t stream_policy = ptx::l2_policy_evict_first();   // dY is read once
         uint32_t phase = 0, idle = 0;
         bool issued = false, ok = true;
@@ -128,24 +150,32 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
         while (__any_sync(0xffffffffu, r < r_end)) {
             bool progressed = false;
             if (r < r_end && ptx::mbar_test_wait(&s_empty[lane], phase ^ 1u)) {
-                s_meta[lane] = make_int4(i_cur, j_cur, __float_as_int(a_cur), 0);
+                const int valid = min(RPS, r_end - r);
+#pragma unroll
+                for (int u = 0; u < RPS; ++u) s_meta[lane][u] = make_int4(i_cur[u], j_cur[u], __float_as_int(a_cur[u]), 0);
                 if (bulk_bytes) {
-                    ptx::mbar_arrive_expect_tx(&s_full[lane], bulk_bytes);
-                    ptx::bulk_load_hint(ring + (size_t)lane * slot_bytes, dY + (int64_t)i_cur * ldy, bulk_bytes, &s_full[lane],
-                                        stream_policy);
+                    ptx::mbar_arrive_expect_tx(&s_full[lane], (uint32_t)valid * bulk_bytes);
+#pragma unroll
+                    for (int u = 0; u < RPS; ++u)
+                        if (u < valid)
+                            ptx::bulk_load_hint(ring + (size_t)lane * slot_bytes + (size_t)u * row_pitch,
+                                                dY + (int64_t)i_cur[u] * ldy, bulk_bytes, &s_full[lane], stream_policy);
                 } else {
                     ptx::mbar_arrive(&s_full[lane]);
                 }
                 issued = true;
                 issued_phase = phase;
                 phase ^= 1u;
-                r += slots;
-                i_cur = i_nxt;
-                if (r < r_end) {
-                    a_cur = alpha[i_cur];
-                    j_cur = f[i_cur];
+                r += round_rows;
+#pragma unroll
+                for (int u = 0; u < RPS; ++u) {
+                    i_cur[u] = i_nxt[u];
+                    if (r + u < r_end) {
+                        a_cur[u] = alpha[i_cur[u]];
+                        j_cur[u] = f[i_cur[u]];
+                    }
+                    i_nxt[u] = r + round_rows + u < r_end ? perm[r + round_rows + u] : -1;
                 }
-                i_nxt = r + slots < r_end ? perm[r + slots] : -1;
                 progressed = true;
             }
             if (__any_sync(0xffffffffu, progressed)) {
@@ -160,7 +190,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                 *abort_flag = 1;
                 raise_status(DEV_TIMEOUT);
             }
-            if (issued) {      // let the copy already issued land before the CTA leaves
+            if (issued) {      // let the copies already issued land before the CTA leaves
                 int never = 0;
                 volatile int* no_abort = &never;
                 ptx::mbar_wait(&s_full[lane], issued_phase, no_abort);
@@ -210,29 +240,46 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
         int slot = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int t = 0; t < nrows; ++t) {
+        for (int t = 0; t < nrows; t += RPS) {
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[slot], phase, abort_flag));   // warp-uniform
             if (!ok) break;
-            const int4 meta = s_meta[slot];
-            const int32_t row = meta.x;
-            const int32_t j = meta.y;
-            const float a = __int_as_float(meta.z);
-            if (j != cur) {
-                if (cur >= 0) flush(cur);
-                cur = j;
-            }
+            const int valid = min(RPS, nrows - t);
             const uint8_t* src = ring + (size_t)slot * slot_bytes;
+            int4 meta[RPS];
+            uint4 raw[RPS][VPT];
 #pragma unroll
-            for (int v = 0; v < VPT; ++v) {
-                const int64_t vec = ct + (int64_t)v * consumers;
-                if (vec < nvec_bulk) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(src + vec * 16);
-                    fma_raw<T>(acc[v], a, raw);
-                } else if (vec < nvec) {     // the ragged last chunk of the row comes straight from global memory
-                    float x[V];
-                    load_vec<T>(dY + (int64_t)row * ldy, vec * V, m, x);
+            for (int u = 0; u < RPS; ++u) {           // every load of the slot first, then the arithmetic
+                meta[u] = s_meta[slot][u];
 #pragma unroll
-                    for (int e = 0; e < V; ++e) acc[v][e] = fmaf(a, x[e], acc[v][e]);
+                for (int v = 0; v < VPT; ++v) {
+                    const int64_t vec = ct + (int64_t)v * consumers;
+                    raw[u][v] = (u < valid && vec < nvec_bulk)
+                                    ? *reinterpret_cast<const uint4*>(src + (size_t)u * row_pitch + vec * 16)
+                                    : make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < RPS; ++u) {
+                if (u < valid) {
+                    const int32_t row = meta[u].x;
+                    const int32_t j = meta[u].y;
+                    const float a = __int_as_float(meta[u].z);
+                    if (j != cur) {
+                        if (cur >= 0) flush(cur);
+                        cur = j;
+                    }
+#pragma unroll
+                    for (int v = 0; v < VPT; ++v) {
+                        const int64_t vec = ct + (int64_t)v * consumers;
+                        if (vec < nvec_bulk) {
+                            fma_raw<T>(acc[v], a, raw[u][v]);
+                        } else if (vec < nvec) {     // the ragged last chunk of the row comes straight from global memory
+                            float x[V];
+                            load_vec<T>(dY + (int64_t)row * ldy, vec * V, m, x);
+#pragma unroll
+                            for (int e = 0; e < V; ++e) acc[v][e] = fmaf(a, x[e], acc[v][e]);
+                        }
+                    }
                 }
             }
             __syncwarp();

@@ -156,13 +156,16 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
         int64_t ranges = std::min<int64_t>(CT_MAX_CTAS, (int64_t)sm_count() * CS_CTAS_PER_SM);
         const int64_t rows_per_cta = std::max<int64_t>(32, (b + ranges - 1) / ranges);
         ranges = (b + rows_per_cta - 1) / rows_per_cta;
-        auto kern = p.vpt == 1 ? contract_stream_kernel<T, 1> : p.vpt == 2 ? contract_stream_kernel<T, 2>
-                                                                           : contract_stream_kernel<T, 4>;
+        auto kern = p.vpt == 4   ? contract_stream_kernel<T, 4, 1>
+                    : p.vpt == 2 ? contract_stream_kernel<T, 2, 1>
+                    : p.rps == 4 ? contract_stream_kernel<T, 1, 4>
+                    : p.rps == 2 ? contract_stream_kernel<T, 1, 2>
+                                 : contract_stream_kernel<T, 1, 1>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
             return PAMM_ERR_CUDA;
         prof_begin(PAMM_PROF_CONTRACT, st);
         launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, alpha, (const T*)dY, ldy, m,
-               (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots, p.slot_bytes,
+               (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots, p.row_pitch,
                p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
         prof_end(PAMM_PROF_CONTRACT, st);
         const int64_t items = k * (w.m_pad / 4);

@@ -30,6 +30,7 @@ SMALL = [
     (5000, 1024, 256, 256, "bf16"),
     (260, 24, 12280, 8, "bf16"),       # dY rows of 24 KiB: four 16-byte chunks per consumer thread
     (96, 16, 24584, 8, "bf16"),        # rows too wide for the shared-memory ring: column-slab path
+    (500, 32, 2600, 12, "bf16"),       # dY rows of 5.2 KB: two rows per ring slot
     (333, 40, 3076, 6, "f32"),         # fp32 rows of 769 chunks: two per consumer thread
 ]
 
