@@ -3,8 +3,10 @@
  *
  * A plain, slow, fp64 CPU statement of what Point-Approximate Matrix
  * Multiplication computes for one linear layer (Algorithm 1 "Compress" and
- * "ApproxMM", Section 3.2, Eq. 1 and Eq. 3 of the paper), at the paper's chosen
- * setting epsilon -> infinity (Section 4.1: no neighbourhood mask, beta = 1).
+ * "ApproxMM", Section 3.2, Eq. 1 and Eq. 3 of the paper).  The paper's chosen
+ * setting is epsilon -> infinity (Section 4.1: no neighbourhood mask, beta = 1);
+ * the neighbourhood condition of Eq. 2 and the factor beta are separate steps
+ * (pamm_oracle_neighbourhood, pamm_oracle_beta) applied after the compression.
  * Only the tests, the smoke check and the benchmark's CPU-baseline leg may call
  * it.  It shares no code, header, table or constant with the CUDA library.
  *
@@ -27,7 +29,10 @@
  * (definition of f below Eq. 1), 1-D line search for alpha, self-representation
  * alpha = 1, orthogonality of the residual, the factorisation C^T B~ = A~^T B
  * with A~ from Eq. 3, k = b identity case equal to the exact A^T B, rank-1 A,
- * the Frobenius error bound of Section 3.2.1, and the printed gamma ~ 28.
+ * the Frobenius error bound of Section 3.2.1, and the printed gamma ~ 28; for the
+ * neighbourhood condition: the equivalent cosine form csim^2 >= 1 - eps^2, eps = 0
+ * against the uniform column-row-sampling estimator, eps >= 1 against eps = infinity,
+ * and the exact unbiasedness of the k = 1, eps = 0 estimate averaged over all rows.
  */
 #include <math.h>
 #include <stdint.h>
@@ -121,6 +126,45 @@ int pamm_oracle_compress(const void *A, int dtype, int64_t b, int64_t n, int64_t
         if (top2_out) top2_out[i] = second;
     }
     return 0;
+}
+
+/* Algorithm 1 "Compress", last two steps, with the neighbourhood condition of Eq. 2:
+ *   e_i = || A_i - alpha_i C_{f(i)} ||_2   (computed from the definition, term by term)
+ *   row i is kept iff e_i <= eps * ||A_i||_2, otherwise alpha_i <- 0 (the row is dropped).
+ * Reading: Algorithm 1 prints the test as "e > eps" (absolute); Eq. 2, the definition in
+ * the text, is relative to ||A_i||; Eq. 2 is followed.  eps = +infinity keeps every row.
+ * alpha is updated in place; kept_out[i] is 1/0, err_out[i] = e_i, rownorm_out[i] = ||A_i||.
+ * Returns eta, the number of dropped rows (Section 3.2, "Normalization factor beta"). */
+int64_t pamm_oracle_neighbourhood(const void *A, int dtype, int64_t b, int64_t n, int64_t lda,
+                                  const double *C, const int32_t *f, double *alpha, double eps,
+                                  uint8_t *kept_out, double *err_out, double *rownorm_out)
+{
+    int64_t i, eta = 0;
+#pragma omp parallel for schedule(static) reduction(+ : eta)
+    for (i = 0; i < b; ++i) {
+        double e2 = 0.0, a2 = 0.0;
+        for (int64_t l = 0; l < n; ++l) {
+            double x = widen(A, dtype, i * lda + l);
+            double r = x - alpha[i] * C[(int64_t)f[i] * n + l];
+            e2 += r * r;
+            a2 += x * x;
+        }
+        double e = sqrt(e2), na = sqrt(a2);
+        int kept = isinf(eps) ? 1 : (e <= eps * na);
+        if (!kept) { alpha[i] = 0.0; eta += 1; }
+        if (kept_out) kept_out[i] = (uint8_t)kept;
+        if (err_out) err_out[i] = e;
+        if (rownorm_out) rownorm_out[i] = na;
+    }
+    return eta;
+}
+
+/* Section 3.2, "Normalization factor beta": beta = b / (b - eta), so that E[O~] = O when
+ * eta rows were dropped (Eq. 4-5).  With every row dropped the estimate is the zero
+ * matrix whatever beta is; 0 is returned then. */
+double pamm_oracle_beta(int64_t b, int64_t eta)
+{
+    return (eta < b) ? (double)b / (double)(b - eta) : 0.0;
 }
 
 /* Algorithm 1 "ApproxMM", first two steps: B' = alpha (.) B and

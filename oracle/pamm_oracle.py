@@ -57,6 +57,10 @@ def _load():
         L.pamm_oracle_weight_grad.restype = None
         L.pamm_oracle_reconstruct.argtypes = [vp, vp, vp, i64, i64, vp]
         L.pamm_oracle_reconstruct.restype = None
+        L.pamm_oracle_neighbourhood.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, ctypes.c_double, vp, vp, vp]
+        L.pamm_oracle_neighbourhood.restype = i64
+        L.pamm_oracle_beta.argtypes = [i64, i64]
+        L.pamm_oracle_beta.restype = ctypes.c_double
         L.pamm_oracle_exact_product.argtypes = [vp, ci, i64, vp, ci, i64, i64, i64, i64, vp]
         L.pamm_oracle_exact_product.restype = None
         L.pamm_oracle_memory_scalars.argtypes = [i64, i64, i64]
@@ -135,6 +139,24 @@ def row_scores(A: np.ndarray, i: int, C: np.ndarray, q: np.ndarray):
     return s, sc, ab
 
 
+def neighbourhood(A: np.ndarray, C: np.ndarray, f: np.ndarray, alpha: np.ndarray, eps: float):
+    """Eq. 2: rows with ||A_i - alpha_i C_f|| > eps ||A_i|| are dropped (alpha_i = 0).
+
+    Returns (alpha_masked, kept, err, rownorm, eta, beta) with beta = b / (b - eta)."""
+    A = _mat(A)
+    C = np.ascontiguousarray(C, np.float64)
+    f = np.ascontiguousarray(f, np.int32)
+    a = np.array(alpha, dtype=np.float64, copy=True)
+    b, n = A.shape
+    kept = np.empty(b, np.uint8)
+    err = np.empty(b, np.float64)
+    rn = np.empty(b, np.float64)
+    L = _load()
+    eta = int(L.pamm_oracle_neighbourhood(_p(A), _dtype_code(A), b, n, _ld(A), _p(C), _p(f), _p(a), float(eps),
+                                          _p(kept), _p(err), _p(rn)))
+    return a, kept.astype(bool), err, rn, eta, float(L.pamm_oracle_beta(b, eta))
+
+
 def contract(f: np.ndarray, alpha: np.ndarray, B: np.ndarray, k: int) -> np.ndarray:
     """B~[j,:] = sum_{i: f_i=j} alpha_i B_i (ApproxMM, index_add step)."""
     B = _mat(B)
@@ -195,10 +217,19 @@ def num_threads() -> int:
     return int(_load().pamm_oracle_num_threads())
 
 
-def pamm(A: np.ndarray, I: np.ndarray, B: np.ndarray):
-    """Whole path given I: returns dict(C, q, f, alpha, top1, top2, Bt, O)."""
+def pamm(A: np.ndarray, I: np.ndarray, B: np.ndarray, eps: float = float("inf")):
+    """Whole path given I: returns dict(C, q, f, alpha, top1, top2, Bt, O) and, for a
+    finite eps, also kept / err / eta / beta with O = beta * C^T B~."""
     C, q = gather(A, I)
     f, alpha, t1, t2 = compress(A, C, q)
+    out = dict(C=C, q=q, f=f, top1=t1, top2=t2)
+    beta = 1.0
+    if np.isfinite(eps):
+        alpha, kept, err, rn, eta, beta = neighbourhood(A, C, f, alpha, eps)
+        out.update(kept=kept, err=err, rownorm=rn, eta=eta, beta=beta)
     Bt = contract(f, alpha, B, C.shape[0])
     O = weight_grad(C, Bt)
-    return dict(C=C, q=q, f=f, alpha=alpha, top1=t1, top2=t2, Bt=Bt, O=O)
+    if beta != 1.0:
+        O = beta * O
+    out.update(alpha=alpha, Bt=Bt, O=O)
+    return out

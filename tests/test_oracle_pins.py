@@ -304,3 +304,82 @@ def test_clustered_data_error_decreases_with_k():
         errs.append(np.linalg.norm(exact - r["O"]) / np.linalg.norm(exact))
     assert errs[0] > errs[1] > errs[2] > errs[3]
     assert errs[3] < 1e-12
+
+
+# ---- neighbourhood condition (Eq. 2) and the factor beta (Eq. 4-5) -----------------------
+
+def test_neighbourhood_matches_cosine_form():
+    """Eq. 2 in its equivalent cosine form: a row is kept iff csim^2 >= 1 - eps^2
+    (from ||A_i - A~_i||^2 = ||A_i||^2 (1 - csim^2), proof of Lemma 1)."""
+    X, dY, I = case(b=400, n=12, k=6, seed=30, centres=8)
+    C, q = orc.gather(X, I)
+    f, alpha, _, _ = orc.compress(X, C, q)
+    X64 = synth.to_f64(X)
+    cs = np.einsum("il,il->i", X64, C[f]) / (np.linalg.norm(X64, axis=1) * np.linalg.norm(C[f], axis=1))
+    for eps in (0.05, 0.2, 0.5, 0.9):
+        a2, kept, err, rn, eta, beta = orc.neighbourhood(X, C, f, alpha, eps)
+        margin = np.abs(cs ** 2 - (1 - eps ** 2))
+        clear = margin > 1e-9
+        assert np.array_equal(kept[clear], (cs ** 2 >= 1 - eps ** 2)[clear])
+        assert 0 < kept.sum() < len(kept)                       # the case exercises both branches
+        assert eta == int((~kept).sum()) and beta == 400 / (400 - eta)
+        assert np.all(a2[~kept] == 0.0) and np.array_equal(a2[kept], alpha[kept])
+        assert np.allclose(rn, np.linalg.norm(X64, axis=1), rtol=1e-13)
+        assert np.allclose(err, np.linalg.norm(X64 - alpha[:, None] * C[f], axis=1), rtol=1e-9, atol=1e-13)
+
+
+def test_epsilon_at_least_one_or_infinite_keeps_everything():
+    X, dY, I = case(b=120, n=10, m=6, k=5, seed=31, centres=0)
+    base = orc.pamm(X, I, dY)
+    for eps in (1.0, 2.5):
+        r = orc.pamm(X, I, dY, eps=eps)
+        assert r["eta"] == 0 and r["beta"] == 1.0 and r["kept"].all()
+        assert np.array_equal(r["alpha"], base["alpha"]) and np.array_equal(r["O"], base["O"])
+    assert "eta" not in base                                    # eps = infinity: the steps are skipped
+
+
+def test_epsilon_zero_is_uniform_column_row_sampling():
+    """Section 4.1: eps = 0 makes PAMM the Uniform-CRS estimator (b/k) A_I^T B_I."""
+    X, dY, I = case(b=90, n=9, m=7, k=10, seed=32, centres=0)     # generic rows: nothing is parallel
+    r = orc.pamm(X, I, dY, eps=0.0)
+    assert np.array_equal(np.nonzero(r["kept"])[0], I) and r["eta"] == 80 and r["beta"] == 9.0
+    crs = (90 / 10) * synth.to_f64(X)[I].T @ synth.to_f64(dY)[I]
+    assert np.allclose(r["O"], crs, rtol=1e-12, atol=1e-14)
+
+
+def test_epsilon_zero_keeps_exact_duplicates_and_multiples():
+    X, dY, I = case(b=60, n=8, m=5, k=3, seed=33, centres=0)
+    X = X.copy()
+    X[50] = X[I[1]]
+    X[51] = -2.0 * X[I[1]]                                        # an exact multiple lies on the generator's line
+    r = orc.pamm(X, I, dY, eps=0.0)
+    assert r["kept"][50] and r["kept"][51] and r["alpha"][51] == -2.0
+    assert r["eta"] == 60 - 5 and abs(r["beta"] - 60 / 5) < 1e-15
+
+
+def test_single_generator_crs_is_exactly_unbiased():
+    """Eq. 5 with k = 1, eps = 0: averaging O~ over every possible choice of the one
+    generator gives sum_i A_i^T B_i = O exactly (beta = b)."""
+    X, dY, _ = case(b=24, n=6, m=4, k=1, seed=34, centres=0)
+    exact = synth.to_f64(X).T @ synth.to_f64(dY)
+    mean = np.zeros_like(exact)
+    for i in range(24):
+        r = orc.pamm(X, np.array([i], np.int32), dY, eps=0.0)
+        assert r["beta"] == 24.0 and r["kept"].sum() == 1
+        mean += r["O"] / 24
+    assert np.allclose(mean, exact, rtol=1e-12, atol=1e-14)
+
+
+def test_kept_set_grows_with_epsilon_and_error_bound_holds():
+    X, dY, I = case(b=300, n=16, m=9, k=8, seed=35, centres=10)
+    prev = None
+    X64, B = synth.to_f64(X), synth.to_f64(dY)
+    for eps in (0.0, 0.1, 0.3, 0.6, 0.95):
+        r = orc.pamm(X, I, dY, eps=eps)
+        if prev is not None:
+            assert np.all(r["kept"] >= prev)
+        prev = r["kept"]
+        # Section 3.2.1: ||O - O~/beta||_F^2 <= ||B||_2^2 (eps^2 ||A_kept||_F^2 + ||A_dropped||_F^2)
+        lhs = np.linalg.norm(X64.T @ B - r["O"] / r["beta"], "fro") ** 2
+        rhs = np.linalg.norm(B, 2) ** 2 * (eps ** 2 * np.sum(X64[r["kept"]] ** 2) + np.sum(X64[~r["kept"]] ** 2))
+        assert lhs <= rhs * (1 + 1e-12) + 1e-18
