@@ -227,9 +227,26 @@ def run_cuda(args):
     ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, dt_code, dev)
     stream = torch.cuda.current_stream()
 
+    eps = args.eps
+    dropped = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def forward(seed):
+        if eps is None:
+            pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+        else:     # neighbourhood condition (Eq. 2): select, then compress with the row-norm warps
+            pamm.select_generators(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, stream=stream)
+            pamm.compress_eps(X, C, invn, eps, f=f, alpha=alpha, dropped=dropped, stream=stream)
+
+    def backward():
+        if eps is None:
+            pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+        else:     # beta = b / (b - eta) applied by the product's epilogue (Eq. 4-5)
+            pamm.contract(f, alpha, dY, k, Btilde=Bt, workspace=ws, stream=stream)
+            pamm.weight_grad_beta(C, Bt, b, dropped, dW=dW, stream=stream)
+
     def step(seed):
-        pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
-        pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+        forward(seed)
+        backward()
 
     for s in range(args.warmup):
         step(w.index_seed + s)
@@ -267,10 +284,10 @@ def run_cuda(args):
         staged = K < PROF_EVERY or s % PROF_EVERY == PROF_EVERY // 2
         if staged:
             ev[s][0].record(stream)
-        pamm.compress_fused(X, k, w.index_seed + s, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+        forward(w.index_seed + s)
         if staged:
             ev[s][1].record(stream)
-        pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+        backward()
         if staged:
             ev[s][2].record(stream)
     t_end.record(stream)
@@ -350,7 +367,8 @@ def run_cuda(args):
         "metric": METRIC, "value": tokens / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world,
         "steps": K, "warmup": args.warmup, "ms_per_step": ms_total / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": f"{w.name}: X {w.dtype} b={b} n={n}, dY b x m={m}, k={k}, per rank",
+        "config": {"workload": f"{w.name}: X {w.dtype} b={b} n={n}, dY b x m={m}, k={k}, per rank"
+                               + ("" if eps is None else f", eps={eps} (dropped {int(dropped.item())} rows)"),
                    "l2": "inputs exceed L2 (X %.0f MiB, dY %.0f MiB per step)" % (b * n * e / 2**20, b * m * e / 2**20)
                    if b * n * e > 126 * 2**20 else "inputs fit L2: warm-cache numbers",
                    "parallelism": f"replicas x{world}"},
@@ -381,6 +399,8 @@ def main():
     ap.add_argument("--ref-budget-s", type=float, default=120.0, help="time budget of the whole --impl reference run")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eps", type=float, default=None,
+                    help="time the neighbourhood-condition path (Eq. 2, beta) with this epsilon instead of epsilon = infinity")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":

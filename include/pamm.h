@@ -6,8 +6,9 @@
  * hidden), B = dY = [dQ|dK|dV] is the upstream gradient (b x m), C holds k
  * generator rows of X, f in [0,k)^b assigns every row to a generator, alpha in
  * R^b scales it, B~ (k x m) is the contracted gradient and dW~ = C^T B~ (n x m)
- * approximates X^T dY.  epsilon = infinity throughout (the paper's chosen
- * setting, Section 4.1): no row is dropped and beta = 1.
+ * approximates X^T dY.  epsilon = infinity (the paper's chosen setting, Section
+ * 4.1: no row is dropped, beta = 1) except in pamm_compress_eps /
+ * pamm_weight_grad_beta, which add the neighbourhood condition and beta.
  *
  * Conventions for every entry point unless its comment says otherwise:
  *  - Matrices are row-major with a leading dimension given in ELEMENTS.
@@ -145,6 +146,38 @@ pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, 
 pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
                              const float* Btilde, int64_t ldb, int64_t m,
                              float* dW, int64_t ldw, void* stream);
+
+/*
+ * Step 2 with the neighbourhood condition (Section 3.2, Eq. 2; Algorithm 1 lines
+ * "e = ||A - alpha (.) C[f,:]||" and "alpha[e > eps] <- 0").  As pamm_compress;
+ * in addition a row whose representative is farther than eps ||X_i|| is dropped,
+ * i.e. gets alpha_i = 0 (f_i is still reported).  The test follows Eq. 2 (relative
+ * to ||X_i||; Algorithm 1 prints it without the norm).  It is evaluated in fp32 as
+ *     ||X_i||^2 - S_{i,f}^2 / ||C_f||^2  <=  (eps^2 + 2 n 2^-24) ||X_i||^2
+ * with ||X_i||^2 summed during the same pass over X: the second term on the right
+ * is the rounding allowance of the two n-term sums, so a row lying exactly on its
+ * generator's line is kept for every eps (eps = 0 is uniform column-row sampling,
+ * Section 4.1), and rows within that allowance of the threshold may fall on either
+ * side of it.  eps >= 1 (or infinite) keeps every row, like pamm_compress.
+ *   eps      >= 0
+ *   dropped  device int32: overwritten with eta, the number of dropped rows
+ */
+pamm_status pamm_compress_eps(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
+                              const void* C, int64_t ldc, int64_t k, const float* c_invnorm, float eps,
+                              int32_t* f, float* alpha, int32_t* dropped,
+                              void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Step 4 with the normalisation factor (Section 3.2, "Normalization factor beta",
+ * Eq. 4-5): dW = beta C^T B~ with beta = b / (b - eta), eta read from `dropped` on
+ * the device when the kernel runs (no host synchronisation).  dropped = NULL means
+ * beta = 1; eta = b (every row dropped) gives dW = 0.
+ *   b        number of rows that were compressed (b of pamm_compress_eps)
+ */
+pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
+                                  const float* Btilde, int64_t ldb, int64_t m,
+                                  int64_t b, const int32_t* dropped,
+                                  float* dW, int64_t ldw, void* stream);
 
 /*
  * Steps 3+4 in one call (Algorithm 3, backward of the linear layer, the

@@ -12,12 +12,16 @@ namespace pamm {
 constexpr int CS_THREADS = 256;
 constexpr int CS_WARPS = CS_THREADS / 32;
 
-template <typename T, int KC>
+// EPS = true adds the neighbourhood condition (Eq. 2): ||X_i||^2 is summed in the same
+// pass and a row with ||X_i||^2 - S^2/||C_f||^2 > (eps^2 + slack) ||X_i||^2 gets alpha = 0;
+// *dropped counts such rows.
+template <typename T, int KC, bool EPS>
 __global__ void __launch_bounds__(CS_THREADS)
 compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
                      const T* __restrict__ C, int64_t ldc, int k,
                      const float* __restrict__ c_invnorm,
-                     int32_t* __restrict__ f, float* __restrict__ alpha) {
+                     int32_t* __restrict__ f, float* __restrict__ alpha, float eps2, float slack,
+                     int32_t* __restrict__ dropped) {
     constexpr int V = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * CS_WARPS + (threadIdx.x >> 5);
@@ -27,7 +31,7 @@ compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
 
     for (int64_t i = warp0; i < b; i += nwarps) {
         const T* xrow = X + i * ldx;
-        float best = -1.f, s_best = 0.f;
+        float best = -1.f, s_best = 0.f, xx = 0.f;
         int j_best = 0;
         for (int j0 = 0; j0 < k; j0 += KC) {
             float acc[KC];
@@ -36,6 +40,10 @@ compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
             for (int64_t col = (int64_t)lane * V; col < n; col += 32 * V) {
                 float x[V];
                 load_vec<T>(xrow, col, n, x);
+                if (EPS && j0 == 0) {
+#pragma unroll
+                    for (int e = 0; e < V; ++e) xx = fmaf(x[e], x[e], xx);
+                }
 #pragma unroll
                 for (int jj = 0; jj < KC; ++jj) {
                     if (j0 + jj < k) {
@@ -63,9 +71,18 @@ compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
                 }
             }
         }
+        if (EPS) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) xx += __shfl_xor_sync(0xffffffffu, xx, off);
+        }
         if (lane == 0) {
+            float a = s_best * __ldg(c_invnorm + k + j_best);
+            if (EPS && xx - s_best * a > (eps2 + slack) * xx) {
+                a = 0.f;
+                atomicAdd(dropped, 1);
+            }
             f[i] = j_best;
-            alpha[i] = s_best * __ldg(c_invnorm + k + j_best);
+            alpha[i] = a;
         }
     }
 }

@@ -12,6 +12,12 @@
 //              with tcgen05.ld and scans them in ascending j with a strict '>'
 //              so the lowest index wins ties; the epilogue of one tile overlaps
 //              the MMAs of the next
+//   warps 6-   (neighbourhood variant only, Eq. 2; four warps per row tile of the
+//              super tile) squared row norms ||X_i||^2: each thread re-reads its
+//              row's 128 bytes of every X tile from shared memory
+//              while the tile waits for / feeds the tensor core, so X is still read
+//              from HBM once; the epilogue then drops a row when
+//              ||X_i||^2 - S^2/||C_f||^2 > eps^2 ||X_i||^2 (+ a rounding allowance)
 // C is small (k x n) and is re-read per row tile from L2; with MT = 2 two row
 // tiles share every C tile.  For k > 256 the generators are processed in chunks
 // with a running (best score, argmax, dot product) per row.
@@ -22,6 +28,7 @@
 namespace pamm {
 
 constexpr int CU_THREADS = 192;
+constexpr int CU_THREADS_EPS(int mt) { return 192 + mt * 128; }   // + one thread per row of the super tile for ||X_i||^2
 constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
 constexpr int CU_TILE_M = 128;
 #ifndef PAMM_CU_BOX_ROWS
@@ -97,14 +104,24 @@ __device__ __forceinline__ void argmax16(const uint32_t (&v)[16], const float* _
     if (sc[0] > best) { best = sc[0]; s_best = sv[0]; j_best = j0 + ji[0]; }
 }
 
-template <int MT>
-__global__ void __launch_bounds__(CU_THREADS, 1)
+// Rounding allowance of the neighbourhood test, relative to ||X_i||^2: both
+// ||X_i||^2 and S^2/||C_f||^2 are fp32 sums of n terms, so their difference is
+// only known to about 2 n 2^-24 ||X_i||^2.  With it, a row that lies exactly on
+// its generator's line (distance 0) is kept for every eps >= 0.
+__host__ __device__ inline float neighbourhood_slack(int64_t n) { return 2.f * (float)n * 5.9604645e-8f; }
+
+// EPS = false: the paper's setting (epsilon = infinity), nothing is dropped.
+// EPS = true : eps2 = epsilon^2 and slack as above; *dropped counts the dropped rows.
+template <int MT, bool EPS>
+__global__ void __launch_bounds__(EPS ? CU_THREADS_EPS(MT) : CU_THREADS, 1)
 compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
                      int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
                      int tmem_cols, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
-                     int32_t* __restrict__ f, float* __restrict__ alpha) {
+                     int32_t* __restrict__ f, float* __restrict__ alpha, float eps2, float slack,
+                     int32_t* __restrict__ dropped) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2];
+    __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2], s_nfull[2], s_nempty[2];
+    __shared__ float s_norm[2][MT * CU_TILE_M];     // ||X_i||^2 of the rows of a super tile (EPS only)
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -122,8 +139,13 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     const int super_rows = MT * CU_TILE_M;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&s_empty[s], 1); }
-        for (int u = 0; u < 2; ++u) { ptx::mbar_init(&s_tfull[u], 1); ptx::mbar_init(&s_tempty[u], 4); }
+        for (int s = 0; s < stages; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&s_empty[s], EPS ? 1 + 4 * MT : 1); }
+        for (int u = 0; u < 2; ++u) {
+            ptx::mbar_init(&s_tfull[u], 1);
+            ptx::mbar_init(&s_tempty[u], 4);
+            ptx::mbar_init(&s_nfull[u], 4 * MT);
+            ptx::mbar_init(&s_nempty[u], 4);
+        }
         s_abort = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async();
@@ -236,6 +258,48 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             }
             if (!ok) raise_status(DEV_TIMEOUT);
         }
+    } else if (EPS && warp >= 6) {
+        // ---------------- squared row norms: one row of the super tile per thread ----------------
+        const int my_mt = (threadIdx.x - 192) / CU_TILE_M, row_in_tile = (threadIdx.x - 192) % CU_TILE_M;
+        const int ksteps_all = num_chunks * ksteps;
+        uint32_t it = 0, sup = 0;
+        bool ok = true;
+        for (int64_t st = r0; st < r1 && ok; st += super_rows, ++sup) {
+            float nrm[4] = {0.f, 0.f, 0.f, 0.f};     // four chains, added at the end in a fixed order
+            const bool live = st + (int64_t)my_mt * CU_TILE_M < r1;
+            for (int q = 0; q < ksteps_all; ++q, ++it) {
+                const int s = it % stages;
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[s], (it / stages) & 1u, abort_flag));   // warp-uniform
+                if (!ok) break;
+                if (q < ksteps && live) {     // the first generator chunk sees every column of X once
+                    const uint8_t* rowp = tiles + (size_t)s * stage_bytes + my_mt * CU_X_TILE_BYTES + row_in_tile * 128;
+                    uint4 w[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)     // chunk c sits at position c ^ (row & 7): conflict-free across the lanes
+                        w[c] = *reinterpret_cast<const uint4*>(rowp + ((c ^ (row_in_tile & 7)) << 4));
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t ws[4] = {w[c].x, w[c].y, w[c].z, w[c].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = bf16_lo(ws[e]), hi = bf16_hi(ws[e]);
+                            nrm[e] = fmaf(lo, lo, nrm[e]);
+                            nrm[e] = fmaf(hi, hi, nrm[e]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&s_empty[s]);     // ordered after this warp's reads of the stage
+            }
+            if (!ok) break;
+            const uint32_t nb = sup & 1u;
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_nempty[nb], ((sup >> 1) & 1u) ^ 1u, abort_flag));
+            if (!ok) break;
+            s_norm[nb][my_mt * CU_TILE_M + row_in_tile] = (nrm[0] + nrm[1]) + (nrm[2] + nrm[3]);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&s_nfull[nb]);
+        }
+        if (!ok && lane == 0) raise_status(DEV_TIMEOUT);
     } else {
         // ---------------- epilogue: one row per thread ----------------
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
@@ -244,9 +308,9 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         for (int j = threadIdx.x - 64; j < kpad; j += 128) s_inv[j] = j < k ? c_invnorm[j] : 0.f;
         for (int j = threadIdx.x - 64; j < k; j += 128) s_inv2[j] = c_invnorm[k + j];
         ptx::named_barrier(1, 128);                      // the four epilogue warps share the norms
-        uint32_t unit = 0;
+        uint32_t unit = 0, sup = 0;
         bool ok = true;
-        for (int64_t st = r0; st < r1 && ok; st += super_rows) {
+        for (int64_t st = r0; st < r1 && ok; st += super_rows, ++sup) {
             float best[MT], s_best[MT];
             int j_best[MT];
 #pragma unroll
@@ -282,14 +346,29 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
             }
+            if (ok && EPS) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_nfull[sup & 1u], (sup >> 1) & 1u, abort_flag));
             if (ok) {
+                int ndrop = 0;
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
                     const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
                     if (row < r1) {
+                        float a = s_best[mt] * s_inv2[j_best[mt]];
+                        if (EPS) {     // Eq. 2: ||X_i - alpha C_f||^2 = ||X_i||^2 - S^2/||C_f||^2 against eps^2 ||X_i||^2
+                            const float nx = s_norm[sup & 1u][mt * CU_TILE_M + quad * 32 + lane];
+                            const float dist2 = nx - s_best[mt] * a;
+                            if (dist2 > (eps2 + slack) * nx) { a = 0.f; ++ndrop; }
+                        }
                         f[row] = j_best[mt];
-                        alpha[row] = s_best[mt] * s_inv2[j_best[mt]];
+                        alpha[row] = a;
                     }
+                }
+                if (EPS) {
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&s_nempty[sup & 1u]);
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) ndrop += __shfl_xor_sync(0xffffffffu, ndrop, off);
+                    if (lane == 0 && ndrop) atomicAdd(dropped, ndrop);
                 }
             }
         }
@@ -306,18 +385,20 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 
 inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
                                         int64_t k, const float* c_invnorm, int32_t* f, float* alpha, int sms,
-                                        bool x_is_ready, cudaStream_t st) {
+                                        bool x_is_ready, cudaStream_t st, bool with_eps = false, float eps = 0.f,
+                                        int32_t* dropped = nullptr) {
     const CompressUmmaPlan p = compress_umma_plan(b, k, sms);
     CUtensorMap tm_x, tm_c;
     if (!make_tmap_bf16_sw128(&tm_x, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, CU_BOX_ROWS) ||
         !make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)p.n_chunk))
         return PAMM_ERR_CUDA;
-    auto kern = p.mt == 2 ? compress_umma_kernel<2> : compress_umma_kernel<1>;
+    auto kern = with_eps ? (p.mt == 2 ? compress_umma_kernel<2, true> : compress_umma_kernel<1, true>)
+                         : (p.mt == 2 ? compress_umma_kernel<2, false> : compress_umma_kernel<1, false>);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
         return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
-    cfg.blockDim = dim3(CU_THREADS);
+    cfg.blockDim = dim3(with_eps ? CU_THREADS_EPS(p.mt) : CU_THREADS);
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -326,7 +407,8 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
-                       p.tmem_cols, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha);
+                       p.tmem_cols, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha, eps * eps,
+                       neighbourhood_slack(n), dropped);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

@@ -28,6 +28,15 @@ __device__ __forceinline__ void raise_status(int bit) { atomicOr(&g_status_word,
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Normalisation factor of Section 3.2 ("Normalization factor beta", Eq. 4-5):
+// beta = b / (b - eta) with eta dropped rows, read from device memory; 1 when no
+// counter is given, 0 when every row was dropped (the estimate is the zero matrix).
+__device__ __forceinline__ float beta_factor(const int32_t* __restrict__ dropped, int64_t b) {
+    if (!dropped) return 1.f;
+    const int64_t eta = *dropped;
+    return eta < b ? (float)((double)b / (double)(b - eta)) : 0.f;
+}
+
 // ---- storage types ----------------------------------------------------------
 template <typename T> struct Vec16;   // 16 bytes of T
 template <> struct Vec16<float> {

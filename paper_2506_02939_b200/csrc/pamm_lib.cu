@@ -101,18 +101,27 @@ pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int6
     return launch_status();
 }
 
+// The neighbourhood condition (Eq. 2) applied or not: eps as given by the caller, the
+// device counter of dropped rows (zeroed on the stream before the kernel).
+struct Neighbourhood {
+    bool on;
+    float eps;
+    int32_t* dropped;
+};
+constexpr Neighbourhood NO_NEIGHBOURHOOD = {false, 0.f, nullptr};
+
 template <typename T>
 pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
-                                 int64_t k, const float* c_invnorm, int32_t* f, float* alpha, cudaStream_t st) {
+                                 int64_t k, const float* c_invnorm, int32_t* f, float* alpha, const Neighbourhood& nb,
+                                 cudaStream_t st) {
     const int64_t want = (b + CS_WARPS - 1) / CS_WARPS;
     const int grid = (int)std::min<int64_t>(want, 148 * 8);
+    const float eps2 = nb.eps * nb.eps, slack = neighbourhood_slack(n);
+    auto kern = nb.on ? (k <= 4 ? compress_simt_kernel<T, 4, true> : compress_simt_kernel<T, 8, true>)
+                      : (k <= 4 ? compress_simt_kernel<T, 4, false> : compress_simt_kernel<T, 8, false>);
     prof_begin(PAMM_PROF_COMPRESS, st);
-    if (k <= 4)
-        launch(compress_simt_kernel<T, 4>, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C,
-               ldc, (int)k, c_invnorm, f, alpha);
-    else
-        launch(compress_simt_kernel<T, 8>, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C,
-               ldc, (int)k, c_invnorm, f, alpha);
+    launch(kern, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C, ldc, (int)k, c_invnorm, f,
+           alpha, eps2, slack, nb.dropped);
     prof_end(PAMM_PROF_COMPRESS, st);
     return launch_status();
 }
@@ -196,11 +205,12 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
 
 template <typename T>
 pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
-                                    int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
+                                    int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows,
+                                    const int32_t* dropped) {
     const int64_t items = n * ((m + 3) / 4);
     prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
     launch(weight_grad_simt_kernel<T>, dim3((unsigned)((items + WG_THREADS - 1) / WG_THREADS)), dim3(WG_THREADS), 0, st, true,
-           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw);
+           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw, b_rows, dropped);
     prof_end(PAMM_PROF_WEIGHT_GRAD, st);
     return launch_status();
 }
@@ -255,36 +265,39 @@ pamm_status check_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, 
 // after our own select kernel), so the compress kernel may read it before that
 // kernel has finished.
 pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
-                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, bool x_is_ready, cudaStream_t st) {
-    if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, bool x_is_ready, cudaStream_t st,
+                        const Neighbourhood& nb = NO_NEIGHBOURHOOD) {
+    if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, nb, st);
     if (compress_umma_supported(b, n, k)) {
         prof_begin(PAMM_PROF_COMPRESS, st);
-        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), x_is_ready, st);
+        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), x_is_ready, st,
+                                                    nb.on, nb.eps, nb.dropped);
         prof_end(PAMM_PROF_COMPRESS, st);
         g_launches += 1;
         return s;
     }
-    return launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, st);
+    return launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, nb, st);
 }
 
 pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
-                           int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
-    if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+                           int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows = 0,
+                           const int32_t* dropped = nullptr) {
+    if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
     if (weight_grad_persist_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st);
+        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
     if (weight_grad_mma_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
-    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st);
+    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
 }
 
 }  // namespace
@@ -390,6 +403,29 @@ pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, p
     pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
     if (s != PAMM_OK) return s;
     return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream);
+}
+
+pamm_status pamm_compress_eps(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C,
+                              int64_t ldc, int64_t k, const float* c_invnorm, float eps, int32_t* f, float* alpha,
+                              int32_t* dropped, void* workspace, size_t ws_bytes, void* stream) {
+    (void)workspace; (void)ws_bytes;
+    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+    if (s != PAMM_OK) return s;
+    if (!dropped || !aligned(dropped, 4) || !(eps >= 0.f)) return PAMM_ERR_INVALID_ARG;     // also rejects NaN
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(dropped, 0, sizeof(int32_t), st) != cudaSuccess) return PAMM_ERR_CUDA;
+    // ||X_i - alpha C_f|| <= ||X_i|| always, so eps >= 1 keeps every row: the plain kernel does
+    const bool on = eps < 1.f;
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, false, st, Neighbourhood{on, eps, dropped});
+}
+
+pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Btilde,
+                                  int64_t ldb, int64_t m, int64_t b, const int32_t* dropped, float* dW, int64_t ldw,
+                                  void* stream) {
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+    if (s != PAMM_OK) return s;
+    if (b < 1 || (dropped && !aligned(dropped, 4))) return PAMM_ERR_INVALID_ARG;
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream, b, dropped);
 }
 
 pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, const int32_t* f, const float* alpha,

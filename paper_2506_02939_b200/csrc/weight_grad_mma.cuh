@@ -39,7 +39,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo_elem, float hi_elem) {
 
 __global__ void __launch_bounds__(WU_THREADS, 2)
 weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* __restrict__ Bt, int64_t ldb,
-                        int k, int n, int m, int kc, int nchunks, float* __restrict__ dW, int64_t ldw) {
+                        int k, int n, int m, int kc, int nchunks, float* __restrict__ dW, int64_t ldw,
+                        int64_t b_rows, const int32_t* __restrict__ dropped) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_tma, s_mma;
     __shared__ uint32_t s_tmem_base;
@@ -139,6 +140,7 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
         // epilogue: thread = one row of the tile; warps 0-3 take columns [0,64), warps 4-7 [64,128)
         const int quad = warp & 3, half = warp >> 2;
         const int64_t row = (int64_t)n0 + quad * 32 + lane;
+        const float beta = beta_factor(dropped, b_rows);
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
             uint32_t v[32];
@@ -150,11 +152,12 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) {
                     if (col + i + 4 <= m) {
-                        *reinterpret_cast<float4*>(out + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                          __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                        *reinterpret_cast<float4*>(out + i) =
+                            make_float4(beta * __uint_as_float(v[i]), beta * __uint_as_float(v[i + 1]),
+                                        beta * __uint_as_float(v[i + 2]), beta * __uint_as_float(v[i + 3]));
                     } else {
                         for (int e = 0; e < 4; ++e)
-                            if (col + i + e < m) out[i + e] = __uint_as_float(v[i + e]);
+                            if (col + i + e < m) out[i + e] = beta * __uint_as_float(v[i + e]);
                     }
                 }
             }
@@ -174,7 +177,8 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
 }
 
 inline pamm_status launch_weight_grad_mma(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
-                                          int64_t m, float* dW, int64_t ldw, cudaStream_t st) {
+                                          int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows = 0,
+                                          const int32_t* dropped = nullptr) {
     const int kpad = (int)round_up(k, 16);
     const int kc = std::min(kpad, WU_KC_MAX);
     const int nchunks = (kpad + kc - 1) / kc;
@@ -194,7 +198,8 @@ inline pamm_status launch_weight_grad_mma(const void* C, int64_t ldc, int64_t k,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, weight_grad_umma_kernel, tm_c, Bt, ldb, (int)k, (int)n, (int)m, kc, nchunks, dW, ldw);
+    cudaLaunchKernelEx(&cfg, weight_grad_umma_kernel, tm_c, Bt, ldb, (int)k, (int)n, (int)m, kc, nchunks, dW, ldw, b_rows,
+                       dropped);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

@@ -41,7 +41,7 @@ inline bool weight_grad_persist_supported(int64_t k, int64_t n, int64_t m) {
 __global__ void __launch_bounds__(WP_THREADS, 1)
 weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_w,
                            const float* __restrict__ Bt, int64_t ldb, int k, int m, int kc, int n_tiles,
-                           int total_tiles, int parts) {
+                           int total_tiles, int parts, int64_t b_rows, const int32_t* __restrict__ dropped) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_afull[2], s_aempty[2], s_tfull[2], s_tempty[2], s_bfull, s_bempty;
     __shared__ uint32_t s_tmem_base;
@@ -154,6 +154,7 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
         const int row = quad * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
+        const float beta = beta_factor(dropped, b_rows);     // Eq. 4-5; 1 unless rows were dropped
         uint32_t it = 0;
         bool ok = true;   // once false this warp only keeps the barrier sequence going
         for (int t = t0; t < t1; ++t, ++it) {
@@ -172,6 +173,10 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
                         uint32_t v[32];
                         ptx::tmem_ld_32x32(tmem_base + lane_base + (uint32_t)(s * WP_TILE + (h * 2 + gg) * 32), v);
                         ptx::tmem_ld_wait();
+                        if (beta != 1.f) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(beta * __uint_as_float(v[i]));
+                        }
                         uint8_t* dst = half + gg * (WP_TILE * 128) + row * 128;
 #pragma unroll
                         for (int c = 0; c < 8; ++c)
@@ -267,7 +272,8 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
 }
 
 inline pamm_status launch_weight_grad_persist(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt,
-                                              int64_t ldb, int64_t m, float* dW, int64_t ldw, int sms, cudaStream_t st) {
+                                              int64_t ldb, int64_t m, float* dW, int64_t ldw, int sms, cudaStream_t st,
+                                              int64_t b_rows = 0, const int32_t* dropped = nullptr) {
     const int kc = (int)round_up(k, 16);
     CUtensorMap tm_c, tm_w;
     if (!make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)kc) ||
@@ -297,7 +303,7 @@ inline pamm_status launch_weight_grad_persist(const void* C, int64_t ldc, int64_
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, weight_grad_persist_kernel, tm_c, tm_w, Bt, ldb, (int)k, (int)m, kc, n_tiles, (int)total,
-                       parts);
+                       parts, b_rows, dropped);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

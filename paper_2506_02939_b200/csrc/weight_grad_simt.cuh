@@ -20,13 +20,14 @@ template <typename T>
 __global__ void __launch_bounds__(WG_THREADS)
 weight_grad_simt_kernel(const T* __restrict__ C, int64_t ldc, int k, int64_t n,
                         const float* __restrict__ Bt, int64_t ldb, int64_t m,
-                        float* __restrict__ dW, int64_t ldw) {
+                        float* __restrict__ dW, int64_t ldw, int64_t b_rows, const int32_t* __restrict__ dropped) {
     const int64_t mv = (m + 3) / 4;
     const int64_t idx = (int64_t)blockIdx.x * WG_THREADS + threadIdx.x;
     grid_dependency_wait();     // B~ (and C) may come from the kernel before
     grid_launch_dependents();
     if (idx >= n * mv) return;
     const int64_t r = idx / mv, col = (idx % mv) * 4;
+    const float beta = beta_factor(dropped, b_rows);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     if (col + 4 <= m) {
         for (int j = 0; j < k; ++j) {
@@ -35,13 +36,13 @@ weight_grad_simt_kernel(const T* __restrict__ C, int64_t ldc, int k, int64_t n,
             acc[0] = fmaf(c, v.x, acc[0]); acc[1] = fmaf(c, v.y, acc[1]);
             acc[2] = fmaf(c, v.z, acc[2]); acc[3] = fmaf(c, v.w, acc[3]);
         }
-        *reinterpret_cast<float4*>(dW + r * ldw + col) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        *reinterpret_cast<float4*>(dW + r * ldw + col) = make_float4(beta * acc[0], beta * acc[1], beta * acc[2], beta * acc[3]);
     } else {
         for (int j = 0; j < k; ++j) {
             const float c = load_scalar<T>(C + (int64_t)j * ldc + r);
             for (int e = 0; e < 4 && col + e < m; ++e) acc[e] = fmaf(c, __ldg(Bt + (int64_t)j * ldb + col + e), acc[e]);
         }
-        for (int e = 0; e < 4 && col + e < m; ++e) dW[r * ldw + col + e] = acc[e];
+        for (int e = 0; e < 4 && col + e < m; ++e) dW[r * ldw + col + e] = beta * acc[e];
     }
 }
 

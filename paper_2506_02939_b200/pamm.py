@@ -37,6 +37,8 @@ _SIGNATURES = {
     "pamm_compress_fused": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_contract": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
     "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
+    "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_weight_grad_beta": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp], _ci),
     "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
     "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
@@ -136,6 +138,29 @@ def compress(X, C, c_invnorm, f=None, alpha=None, workspace=None, stream=None):
     _check(_lib.pamm_compress(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), _ptr(f),
                               _ptr(alpha), _ptr(workspace), ws_bytes, _stream(stream)), "pamm_compress")
     return f, alpha
+
+
+def compress_eps(X, C, c_invnorm, eps: float, f=None, alpha=None, dropped=None, stream=None):
+    """compress with the neighbourhood condition (Eq. 2): rows farther than eps ||X_i|| from their representative
+    get alpha = 0; ``dropped`` (device int32[1]) receives their number."""
+    b, n = X.shape
+    k = C.shape[0]
+    f = torch.empty(b, dtype=torch.int32, device=X.device) if f is None else f
+    alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
+    dropped = torch.empty(1, dtype=torch.int32, device=X.device) if dropped is None else dropped
+    _check(_lib.pamm_compress_eps(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), float(eps), _ptr(f),
+                                  _ptr(alpha), _ptr(dropped), None, 0, _stream(stream)), "pamm_compress_eps")
+    return f, alpha, dropped
+
+
+def weight_grad_beta(C, Btilde, b: int, dropped, dW=None, stream=None):
+    """dW = beta C^T B~ with beta = b / (b - eta), eta read from ``dropped`` on the device (Eq. 4-5)."""
+    k, n = C.shape
+    m = Btilde.shape[1]
+    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
+    _check(_lib.pamm_weight_grad_beta(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, b, _ptr(dropped),
+                                      _ptr(dW), _ld(dW), _stream(stream)), "pamm_weight_grad_beta")
+    return dW
 
 
 def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, f=None, alpha=None,
