@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use: mbarrier,
-// TMA tile loads (cp.async.bulk.tensor, never multicast), tensor memory (TMEM)
+// TMA tile loads (cp.async.bulk.tensor, each CTA fetching its own tiles), tensor memory (TMEM)
 // allocation, tcgen05.mma / commit / ld, and the UMMA descriptors.
 // Every wait is bounded: it gives up after a fixed number of polls and reports
 // false so the caller can raise the status word and leave in an orderly way.
