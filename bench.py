@@ -387,6 +387,87 @@ def run_cuda(args):
     print(json.dumps(line), flush=True)
 
 
+def run_layer_loop(args):
+    """A stack of QKV layers on one GPU: every layer's forward compress keeps only (C, f, alpha),
+    then the backward passes run in reverse order.  Reports tokens/s per layer and the bytes kept
+    for the backward pass against storing every layer's X (the memory the method is about)."""
+    import torch
+    from paper_2506_02939_b200 import build as pamm_build, synth
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the PAMM path has no CPU fallback")
+    torch.cuda.set_device(env_int("LOCAL_RANK", 0))
+    pamm_build.build()
+    from paper_2506_02939_b200 import pamm
+    w = synth.WORKLOADS[args.workload]
+    k = args.k or w.ks[0]
+    L = args.layers
+    e = 2 if w.dtype == "bf16" else 4
+    dt_code = pamm.BF16 if w.dtype == "bf16" else pamm.F32
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    D = min(L, args.distinct_layers)      # distinct input sets (seed + 100 * layer), reused cyclically
+
+    def dev(a):
+        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return t.cuda()
+
+    Xs, dYs = [], []
+    for d in range(D):
+        inp = synth.make_inputs(args.workload, seed=w.seed + 100 * d)
+        Xs.append(dev(inp.X))
+        dYs.append(dev(inp.dY))
+    b, n, m = w.b, w.n, w.m
+    devc = Xs[0].device
+    saved = [dict(idx=torch.empty(k, dtype=torch.int32, device=devc), C=torch.empty((k, n), dtype=tdt, device=devc),
+                  invn=torch.empty(2 * k, dtype=torch.float32, device=devc),
+                  f=torch.empty(b, dtype=torch.int32, device=devc), alpha=torch.empty(b, dtype=torch.float32, device=devc))
+             for _ in range(L)]
+    dW = torch.empty((n, m), dtype=torch.float32, device=devc)
+    ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, dt_code, devc)
+    stream = torch.cuda.current_stream()
+
+    def step(s):
+        for l in range(L):
+            sv = saved[l]
+            pamm.compress_fused(Xs[l % D], k, w.index_seed + 100 * l + s, idx_out=sv["idx"], C=sv["C"], c_invnorm=sv["invn"],
+                                f=sv["f"], alpha=sv["alpha"], stream=stream)
+        for l in reversed(range(L)):
+            sv = saved[l]
+            pamm.contract_weight_grad(sv["C"], sv["f"], sv["alpha"], dYs[l % D], dW=dW, workspace=ws, stream=stream)
+
+    for s in range(max(3, args.warmup)):
+        step(s)
+    torch.cuda.synchronize()
+    K = max(1, args.steps)
+    sampler = ClockSampler(env_int("LOCAL_RANK", 0))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = pamm.launch_count()
+    sampler.start()
+    e0.record(stream)
+    for s in range(K):
+        step(s)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    status = pamm.last_device_status()
+    if status != pamm.OK:
+        raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
+    ms = e0.elapsed_time(e1)
+    kept = sum(sum(t.numel() * t.element_size() for key, t in sv.items() if key in ("C", "f", "alpha")) for sv in saved)
+    full = L * b * n * e
+    line = {
+        "metric": METRIC, "value": b * L * K / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": K,
+        "warmup": max(3, args.warmup), "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": f"{w.name} x {L} layers: X {w.dtype} b={b} n={n}, dY b x m={m}, k={k}; forward of all layers, "
+                               f"then backward in reverse; {D} distinct input sets (seed + 100 * layer) reused cyclically",
+                   "l2": "inputs exceed L2"},
+        "memory_saved": {"layers": L, "kept_bytes_all_layers": int(kept), "x_bytes_all_layers": int(full), "ratio": full / kept,
+                         "scalars_kept": L * (k * n + 2 * b), "scalars_x": L * b * n},
+        "gpu_launches": int(pamm.launch_count() - launches0), "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -401,10 +482,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eps", type=float, default=None,
                     help="time the neighbourhood-condition path (Eq. 2, beta) with this epsilon instead of epsilon = infinity")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="with L > 1: a stack of L layers (forward of all, then backward in reverse) and its saved-activation bytes")
+    ap.add_argument("--distinct-layers", type=int, default=4, help="distinct synthetic input sets in the --layers mode")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.layers > 1:
+        run_layer_loop(args)
     else:
         run_cuda(args)
     import torch.distributed as dist

@@ -220,3 +220,32 @@ def test_workload_c3_ratio_sweep():
     for k in w.ks:
         rep = parity.run_and_compare(inp.X, inp.dY, k, seed=w.index_seed)
         print("c3", k, rep.err, "mismatch", rep.mismatches, "near-tie", rep.near_tie, "rounding", rep.explained_by_rounding)
+
+
+def test_layer_stack_keeps_only_the_compressed_state():
+    """c5-shaped layers at reduced batch: forward of every layer first (X is not needed afterwards),
+    backward in reverse order from the kept (C, f, alpha) only; the bytes kept follow k n e + 8 b."""
+    L = 3
+    layers = [synth.make_inputs("c5", num_seqs=1, seed=4 + 100 * l) for l in range(L)]
+    w = layers[0].workload
+    b, n, m, k = layers[0].b, w.n, w.m, w.ks[0]
+    kept = []
+    for l, inp in enumerate(layers):
+        Xd = parity.to_device(inp.X)
+        idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, w.index_seed + 100 * l)
+        kept.append((idx, C, f, alpha))
+        del Xd                                                     # the layer's input is gone after its forward pass
+    kept_bytes = sum(C.numel() * 2 + f.numel() * 4 + alpha.numel() * 4 for _, C, f, alpha in kept)
+    assert kept_bytes == L * (k * n * 2 + 8 * b)
+    assert pamm.saved_bytes(b, n, k, pamm.BF16)["pamm"] * L == kept_bytes
+    assert L * b * n * 2 / kept_bytes > 100                        # 341x at the full batch, 114x at this one
+    rng = np.random.default_rng(0)
+    rr, cc = rng.integers(0, n, 2048), rng.integers(0, m, 2048)
+    for l in reversed(range(L)):
+        idx, C, f, alpha = kept[l]
+        dW = pamm.contract_weight_grad(C, f, alpha, parity.to_device(layers[l].dY)).cpu().numpy()
+        assert pamm.last_device_status() == pamm.OK
+        C64 = synth.to_f64(parity.from_device_bits(C))
+        Bt = orc.contract(f.cpu().numpy(), alpha.cpu().numpy().astype(np.float64), layers[l].dY, k)
+        ref = np.einsum("js,js->s", C64[:, rr], Bt[:, cc])
+        assert parity.rel_fro(dW[rr, cc], ref) <= 1e-2
