@@ -46,6 +46,7 @@ struct CompressUmmaPlan {
     int stages;
     int stage_bytes;
     int tmem_cols;
+    int tmem_bufs;
     int rows_per_cta;
     int grid;
     size_t smem_bytes;
@@ -60,10 +61,15 @@ inline CompressUmmaPlan compress_umma_plan(int64_t b, int64_t k, int sms) {
     const int npad = (int)round_up(k, 16);
     p.num_chunks = (npad + 255) / 256;
     p.n_chunk = (int)round_up((npad + p.num_chunks - 1) / p.num_chunks, 16);
+#ifdef PAMM_CU_MT1_WIDE
     p.mt = p.n_chunk <= 128 ? 2 : 1;
+#else
+    p.mt = 2;      // two row tiles share every C tile; beyond 128 generators per chunk they fill TMEM (one buffer)
+#endif
     p.stage_bytes = p.mt * CU_X_TILE_BYTES + p.n_chunk * 128;
     p.stages = std::min(8, CU_SMEM_BUDGET / p.stage_bytes);
-    int cols = 2 * p.mt * p.n_chunk;
+    p.tmem_bufs = 2 * p.mt * p.n_chunk <= 512 ? 2 : 1;     // accumulator sets: the epilogue overlaps the next MMAs only with two
+    int cols = p.tmem_bufs * p.mt * p.n_chunk;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols *= 2;
     const int64_t per = (b + sms - 1) / sms;
@@ -116,7 +122,7 @@ template <int MT, bool EPS>
 __global__ void __launch_bounds__(EPS ? CU_THREADS_EPS(MT) : CU_THREADS, 1)
 compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
                      int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
-                     int tmem_cols, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
+                     int tmem_cols, int tmem_bufs, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
                      int32_t* __restrict__ f, float* __restrict__ alpha, float eps2, float slack,
                      int32_t* __restrict__ dropped) {
     extern __shared__ uint8_t smem_raw[];
@@ -232,7 +238,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             bool ok = true;
             for (int64_t st = r0; st < r1 && ok; st += super_rows) {
                 for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
-                    const uint32_t buf = unit & 1u, uph = (unit >> 1) & 1u;
+                    const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
                     if (!ptx::mbar_wait(&s_tempty[buf], uph ^ 1u, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     const uint32_t d_base = tmem_base + buf * (uint32_t)(MT * n_chunk);
@@ -316,7 +322,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 #pragma unroll
             for (int mt = 0; mt < MT; ++mt) { best[mt] = -1.f; s_best[mt] = 0.f; j_best[mt] = 0; }
             for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
-                const uint32_t buf = unit & 1u, uph = (unit >> 1) & 1u;
+                const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_tfull[buf], uph, abort_flag));   // warp-uniform
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
@@ -407,7 +413,7 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
-                       p.tmem_cols, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha, eps * eps,
+                       p.tmem_cols, p.tmem_bufs, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha, eps * eps,
                        neighbourhood_slack(n), dropped);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
