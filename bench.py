@@ -33,7 +33,7 @@ PROF_EVERY = 16     # one step in PROF_EVERY carries per-kernel CUDA events, ano
                     # the rest run event-free, since an event between two kernels serialises their launches
 # DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
 # summarised under profiles/, keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {"c4": 812307456}     # contract_stream_kernel<bf16,2>: 806.12 MB read + 6.19 MB written
+NCU_TRAFFIC_BYTES = {"c4": 811204096}     # contract_stream_kernel<bf16,2,1>: 806.14 MB read + 5.06 MB written
 
 
 def env_int(name, default):
