@@ -180,6 +180,15 @@ pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t
                                   float* dW, int64_t ldw, void* stream);
 
 /*
+ * Step 4, accumulating: dW += C^T B~ (Algorithm 3's weight gradient added to what dW
+ * already holds, as gradient accumulation over micro-batches needs).  Every element
+ * of dW receives exactly one addition per call, so the result is reproducible.
+ */
+pamm_status pamm_weight_grad_accumulate(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
+                                        const float* Btilde, int64_t ldb, int64_t m,
+                                        float* dW, int64_t ldw, void* stream);
+
+/*
  * Steps 3+4 in one call (Algorithm 3, backward of the linear layer, the
  * weight-gradient half): contract dY into B~ and multiply by C^T.  Btilde may
  * be NULL, in which case B~ lives in the workspace only.

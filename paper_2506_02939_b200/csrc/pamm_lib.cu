@@ -206,11 +206,11 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
 template <typename T>
 pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
                                     int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows,
-                                    const int32_t* dropped) {
+                                    const int32_t* dropped, bool accumulate) {
     const int64_t items = n * ((m + 3) / 4);
     prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
     launch(weight_grad_simt_kernel<T>, dim3((unsigned)((items + WG_THREADS - 1) / WG_THREADS)), dim3(WG_THREADS), 0, st, true,
-           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw, b_rows, dropped);
+           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw, b_rows, dropped, accumulate ? 1 : 0);
     prof_end(PAMM_PROF_WEIGHT_GRAD, st);
     return launch_status();
 }
@@ -281,23 +281,25 @@ pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_d
 
 pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
                            int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows = 0,
-                           const int32_t* dropped = nullptr) {
-    if (dt == PAMM_F32) return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
+                           const int32_t* dropped = nullptr, bool accumulate = false) {
+    if (dt == PAMM_F32)
+        return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
     if (weight_grad_persist_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped);
+        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped,
+                                                          accumulate);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
     if (weight_grad_mma_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
+        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
-    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped);
+    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
 }
 
 }  // namespace
@@ -426,6 +428,13 @@ pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t
     if (s != PAMM_OK) return s;
     if (b < 1 || (dropped && !aligned(dropped, 4))) return PAMM_ERR_INVALID_ARG;
     return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream, b, dropped);
+}
+
+pamm_status pamm_weight_grad_accumulate(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
+                                        const float* Btilde, int64_t ldb, int64_t m, float* dW, int64_t ldw, void* stream) {
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+    if (s != PAMM_OK) return s;
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream, 0, nullptr, true);
 }
 
 pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, const int32_t* f, const float* alpha,

@@ -40,7 +40,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo_elem, float hi_elem) {
 __global__ void __launch_bounds__(WU_THREADS, 2)
 weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* __restrict__ Bt, int64_t ldb,
                         int k, int n, int m, int kc, int nchunks, float* __restrict__ dW, int64_t ldw,
-                        int64_t b_rows, const int32_t* __restrict__ dropped) {
+                        int64_t b_rows, const int32_t* __restrict__ dropped, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_tma, s_mma;
     __shared__ uint32_t s_tmem_base;
@@ -152,12 +152,16 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) {
                     if (col + i + 4 <= m) {
-                        *reinterpret_cast<float4*>(out + i) =
-                            make_float4(beta * __uint_as_float(v[i]), beta * __uint_as_float(v[i + 1]),
-                                        beta * __uint_as_float(v[i + 2]), beta * __uint_as_float(v[i + 3]));
+                        float4 o = make_float4(beta * __uint_as_float(v[i]), beta * __uint_as_float(v[i + 1]),
+                                               beta * __uint_as_float(v[i + 2]), beta * __uint_as_float(v[i + 3]));
+                        if (accumulate) {
+                            const float4 old = *reinterpret_cast<const float4*>(out + i);
+                            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                        }
+                        *reinterpret_cast<float4*>(out + i) = o;
                     } else {
                         for (int e = 0; e < 4; ++e)
-                            if (col + i + e < m) out[i + e] = beta * __uint_as_float(v[i + e]);
+                            if (col + i + e < m) out[i + e] = beta * __uint_as_float(v[i + e]) + (accumulate ? out[i + e] : 0.f);
                     }
                 }
             }
@@ -178,7 +182,7 @@ weight_grad_umma_kernel(const __grid_constant__ CUtensorMap tm_c, const float* _
 
 inline pamm_status launch_weight_grad_mma(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
                                           int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows = 0,
-                                          const int32_t* dropped = nullptr) {
+                                          const int32_t* dropped = nullptr, bool accumulate = false) {
     const int kpad = (int)round_up(k, 16);
     const int kc = std::min(kpad, WU_KC_MAX);
     const int nchunks = (kpad + kc - 1) / kc;
@@ -199,7 +203,7 @@ inline pamm_status launch_weight_grad_mma(const void* C, int64_t ldc, int64_t k,
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, weight_grad_umma_kernel, tm_c, Bt, ldb, (int)k, (int)n, (int)m, kc, nchunks, dW, ldw, b_rows,
-                       dropped);
+                       dropped, accumulate ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

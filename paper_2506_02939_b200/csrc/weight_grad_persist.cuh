@@ -41,7 +41,8 @@ inline bool weight_grad_persist_supported(int64_t k, int64_t n, int64_t m) {
 __global__ void __launch_bounds__(WP_THREADS, 1)
 weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_w,
                            const float* __restrict__ Bt, int64_t ldb, int k, int m, int kc, int n_tiles,
-                           int total_tiles, int parts, int64_t b_rows, const int32_t* __restrict__ dropped) {
+                           int total_tiles, int parts, int64_t b_rows, const int32_t* __restrict__ dropped,
+                           int accumulate) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_afull[2], s_aempty[2], s_tfull[2], s_tempty[2], s_bfull, s_bempty;
     __shared__ uint32_t s_tmem_base;
@@ -192,9 +193,12 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
                 ptx::fence_proxy_async();
                 ptx::named_barrier(WP_EPI_BARRIER, WP_EPI_THREADS);
                 if (etid == 0) {
-                    if (ok) {
+                    if (ok && !accumulate) {
                         ptx::tma_store_2d(&tm_w, half, m0 + h * 64, n0);
                         ptx::tma_store_2d(&tm_w, half + WP_TILE * 128, m0 + h * 64 + 32, n0);
+                    } else if (ok) {     // dW += tile (gradient accumulation)
+                        ptx::tma_reduce_add_2d(&tm_w, half, m0 + h * 64, n0);
+                        ptx::tma_reduce_add_2d(&tm_w, half + WP_TILE * 128, m0 + h * 64 + 32, n0);
                     }
                     ptx::bulk_commit_group();
                 }
@@ -273,7 +277,7 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
 
 inline pamm_status launch_weight_grad_persist(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt,
                                               int64_t ldb, int64_t m, float* dW, int64_t ldw, int sms, cudaStream_t st,
-                                              int64_t b_rows = 0, const int32_t* dropped = nullptr) {
+                                              int64_t b_rows = 0, const int32_t* dropped = nullptr, bool accumulate = false) {
     const int kc = (int)round_up(k, 16);
     CUtensorMap tm_c, tm_w;
     if (!make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)kc) ||
@@ -303,7 +307,7 @@ inline pamm_status launch_weight_grad_persist(const void* C, int64_t ldc, int64_
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, weight_grad_persist_kernel, tm_c, tm_w, Bt, ldb, (int)k, (int)m, kc, n_tiles, (int)total,
-                       parts, b_rows, dropped);
+                       parts, b_rows, dropped, accumulate ? 1 : 0);
     return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
 }
 

@@ -20,7 +20,8 @@ template <typename T>
 __global__ void __launch_bounds__(WG_THREADS)
 weight_grad_simt_kernel(const T* __restrict__ C, int64_t ldc, int k, int64_t n,
                         const float* __restrict__ Bt, int64_t ldb, int64_t m,
-                        float* __restrict__ dW, int64_t ldw, int64_t b_rows, const int32_t* __restrict__ dropped) {
+                        float* __restrict__ dW, int64_t ldw, int64_t b_rows, const int32_t* __restrict__ dropped,
+                        int accumulate) {
     const int64_t mv = (m + 3) / 4;
     const int64_t idx = (int64_t)blockIdx.x * WG_THREADS + threadIdx.x;
     grid_dependency_wait();     // B~ (and C) may come from the kernel before
@@ -36,13 +37,19 @@ weight_grad_simt_kernel(const T* __restrict__ C, int64_t ldc, int k, int64_t n,
             acc[0] = fmaf(c, v.x, acc[0]); acc[1] = fmaf(c, v.y, acc[1]);
             acc[2] = fmaf(c, v.z, acc[2]); acc[3] = fmaf(c, v.w, acc[3]);
         }
-        *reinterpret_cast<float4*>(dW + r * ldw + col) = make_float4(beta * acc[0], beta * acc[1], beta * acc[2], beta * acc[3]);
+        float4 o = make_float4(beta * acc[0], beta * acc[1], beta * acc[2], beta * acc[3]);
+        if (accumulate) {
+            const float4 old = *reinterpret_cast<const float4*>(dW + r * ldw + col);
+            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+        }
+        *reinterpret_cast<float4*>(dW + r * ldw + col) = o;
     } else {
         for (int j = 0; j < k; ++j) {
             const float c = load_scalar<T>(C + (int64_t)j * ldc + r);
             for (int e = 0; e < 4 && col + e < m; ++e) acc[e] = fmaf(c, __ldg(Bt + (int64_t)j * ldb + col + e), acc[e]);
         }
-        for (int e = 0; e < 4 && col + e < m; ++e) dW[r * ldw + col + e] = beta * acc[e];
+        for (int e = 0; e < 4 && col + e < m; ++e)
+            dW[r * ldw + col + e] = beta * acc[e] + (accumulate ? dW[r * ldw + col + e] : 0.f);
     }
 }
 

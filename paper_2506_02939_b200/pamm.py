@@ -39,6 +39,7 @@ _SIGNATURES = {
     "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
     "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_weight_grad_beta": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp], _ci),
+    "pamm_weight_grad_accumulate": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
     "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
     "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
@@ -160,6 +161,15 @@ def weight_grad_beta(C, Btilde, b: int, dropped, dW=None, stream=None):
     dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
     _check(_lib.pamm_weight_grad_beta(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, b, _ptr(dropped),
                                       _ptr(dW), _ld(dW), _stream(stream)), "pamm_weight_grad_beta")
+    return dW
+
+
+def weight_grad_accumulate(C, Btilde, dW, stream=None):
+    """dW += C^T B~ (gradient accumulation over micro-batches)."""
+    k, n = C.shape
+    m = Btilde.shape[1]
+    _check(_lib.pamm_weight_grad_accumulate(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW),
+                                            _stream(stream)), "pamm_weight_grad_accumulate")
     return dW
 
 

@@ -249,3 +249,19 @@ def test_layer_stack_keeps_only_the_compressed_state():
         Bt = orc.contract(f.cpu().numpy(), alpha.cpu().numpy().astype(np.float64), layers[l].dY, k)
         ref = np.einsum("js,js->s", C64[:, rr], Bt[:, cc])
         assert parity.rel_fro(dW[rr, cc], ref) <= 1e-2
+
+
+@pytest.mark.parametrize("k,n,m,dtype", [(24, 136, 264, "bf16"), (200, 72, 136, "bf16"), (5, 40, 52, "f32")])
+def test_weight_grad_accumulate_adds_to_dW(k, n, m, dtype):
+    # the three product kernels (persistent tcgen05, one-tile tcgen05, CUDA cores): dW += C^T B~, twice
+    Cb, _ = synth.random_case(k, n, 8, dtype, seed=21)
+    Bt = torch.from_numpy(np.random.default_rng(22).standard_normal((k, m)).astype(np.float32)).cuda()
+    C = parity.to_device(Cb)
+    base = torch.from_numpy(np.random.default_rng(23).standard_normal((n, m)).astype(np.float32)).cuda()
+    once = pamm.weight_grad(C, Bt)
+    dW = base.clone()
+    pamm.weight_grad_accumulate(C, Bt, dW)
+    assert torch.allclose(dW, base + once, rtol=1e-6, atol=1e-6)
+    pamm.weight_grad_accumulate(C, Bt, dW)
+    assert torch.allclose(dW, base + 2 * once, rtol=1e-6, atol=1e-5)
+    assert pamm.last_device_status() == pamm.OK
