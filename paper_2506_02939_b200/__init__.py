@@ -4,4 +4,4 @@
 import when the library has not been built; ``paper_2506_02939_b200.synth``
 makes seeded synthetic inputs and needs numpy only.
 """
-__all__ = ["pamm", "synth"]
+__all__ = ["pamm", "synth", "autograd"]

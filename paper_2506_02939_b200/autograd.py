@@ -1,0 +1,65 @@
+"""A linear layer whose backward pass keeps the compressed input only (Algorithms 2 and 3).
+
+Forward: ``Z = X W`` (an ordinary GEMM, done by torch) and ``Compress(flatten(X))`` through
+the CUDA library; the layer saves (C, f, alpha, W) and lets go of X.  Backward: the weight
+gradient is ``ApproxMM(C, alpha, f, dZ) = C^T B~`` through the library, the input gradient
+``dX = dZ W^T`` is exact (torch).  Meant for the fused Q|K|V projection: ``W`` is n x m
+with m = |Q| + |K| + |V|, as in the paper's notation.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from . import pamm
+
+
+def _rows(t: torch.Tensor, cols: int) -> torch.Tensor:
+    """(…, cols) -> contiguous (rows, cols) view the library accepts (16-byte aligned rows)."""
+    t2 = t.reshape(-1, cols)
+    if t2.stride(1) != 1 or (t2.stride(0) * t2.element_size()) % 16 or t2.data_ptr() % 16:
+        padded = pamm.alloc_matrix(t2.shape[0], cols, t2.dtype, t2.device)
+        padded.copy_(t2)
+        t2 = padded
+    return t2
+
+
+class PammLinearFunction(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, X, W, k, seed):
+        n, m = W.shape
+        Z = X @ W
+        X2 = _rows(X.detach(), n)
+        _, C, _, f, alpha = pamm.compress_fused(X2, int(k), int(seed))
+        ctx.save_for_backward(C, f, alpha, W)          # k n + 2 b scalars instead of b n
+        return Z
+
+    @staticmethod
+    def backward(ctx, dZ):
+        C, f, alpha, W = ctx.saved_tensors
+        n, m = W.shape
+        dX = dZ @ W.t() if ctx.needs_input_grad[0] else None
+        dW = None
+        if ctx.needs_input_grad[1]:
+            dZ2 = _rows(dZ.to(C.dtype), m)
+            dW = pamm.contract_weight_grad(C, f, alpha, dZ2).to(W.dtype)
+        return dX, dW, None, None
+
+
+class PammLinear(torch.nn.Module):
+    """``Z = X W`` with PAMM in the backward pass; ``r`` is the compression ratio k / b (Section 4.1)."""
+
+    def __init__(self, n: int, m: int, r: float = 1.0 / 512, dtype=torch.bfloat16, device="cuda", seed: int = 0):
+        super().__init__()
+        self.weight = torch.nn.Parameter(torch.empty((n, m), dtype=dtype, device=device))
+        torch.nn.init.normal_(self.weight, std=1.0 / math.sqrt(n))
+        self.r = float(r)
+        self.seed = int(seed)
+        self.calls = 0
+
+    def forward(self, X):
+        b = X.numel() // X.shape[-1]
+        k = max(1, min(b, math.ceil(self.r * b)))
+        self.calls += 1                                   # fresh generators every step (Appendix "LLaMA-1B Runtime Breakdown")
+        return PammLinearFunction.apply(X, self.weight, k, self.seed + self.calls)
