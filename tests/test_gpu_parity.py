@@ -43,6 +43,20 @@ def test_small_cases(b, n, m, k, dtype, fused):
     assert rep.unexplained == 0
 
 
+def test_many_rows_ragged_everywhere():
+    # more rows than 148 x 1024 (several sort blocks per SM, ranges of ~1350 rows per CTA), nothing a multiple of a tile
+    X, dY = synth.random_case(200003, 264, 520, "bf16", seed=51, centres=40, dy_scale=1e-3)
+    rep = parity.run_and_compare(X, dY, 96, seed=52, full_dW=False)
+    assert rep.unexplained == 0
+
+
+def test_largest_generator_count_of_the_tensor_core_path():
+    # k = 4096: sixteen chunks of 256 generators with a running argmax per row; k = 4097 takes the CUDA-core path
+    X, dY = synth.random_case(4500, 128, 72, "bf16", seed=53, centres=300, dy_scale=1e-3)
+    parity.run_and_compare(X, dY, 4096, seed=54, full_dW=False)
+    parity.run_and_compare(X[:4200], dY[:4200], 4097, seed=55, full_dW=False)
+
+
 def test_ragged_columns_with_padded_leading_dimension():
     # n and m are not multiples of the 16-byte vector; the row stride is
     X, dY = synth.random_case(700, 70, 45, "f32", seed=3, centres=6)
