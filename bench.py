@@ -292,11 +292,23 @@ def run_cuda(args):
             ev[s][2].record(stream)
     t_end.record(stream)
     torch.cuda.synchronize()
+    launches = pamm.launch_count() - launches0
     barrier()
+    covers = "timed region"
+    if t_begin.elapsed_time(t_end) < 500.0:
+        # a region this short yields too few 50 ms samples: keep sampling over an untimed repeat of the same steps
+        covers = "timed region + untimed repeat of it (region shorter than 0.5 s)"
+        for kind in kev:
+            pamm.set_profile_events(kind, None, None)
+        t_rep = time.perf_counter()
+        while time.perf_counter() - t_rep < 0.5:
+            for s in range(16):
+                step(w.index_seed + s)
+            torch.cuda.synchronize()
     clocks = sampler.stop()
+    clocks["covers"] = covers
     for kind in kev:
         pamm.set_profile_events(kind, None, None)
-    launches = pamm.launch_count() - launches0
     status = pamm.last_device_status()
     if status != pamm.OK:
         raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
@@ -471,8 +483,8 @@ def run_layer_loop(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 2000; 20 for --impl reference)")
+    ap.add_argument("--warmup", type=int, default=None, help="untimed steps (default 20; 2 for --impl reference)")
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="c4", help="c1..c5; c4 (LLaMA-1B-shaped) is the headline configuration")
     ap.add_argument("--k", type=int, default=0, help="override the workload's generator count")
@@ -486,7 +498,12 @@ def main():
                     help="with L > 1: a stack of L layers (forward of all, then backward in reverse) and its saved-activation bytes")
     ap.add_argument("--distinct-layers", type=int, default=4, help="distinct synthetic input sets in the --layers mode")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.steps is None:
+        args.steps = 2000 if args.impl == "cuda" else 20
+    if args.warmup is None:
+        args.warmup = 20 if args.impl == "cuda" else 2
+    if args.impl == "cuda":
+        args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
     elif args.layers > 1:
