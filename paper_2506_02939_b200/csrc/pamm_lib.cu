@@ -14,8 +14,8 @@
 #include "contract.cuh"
 #include "contract_stream.cuh"
 #include "weight_grad_simt.cuh"
-#include "weight_grad_mma.cuh"
 #include "weight_grad_persist.cuh"
+#include "weight_grad_chunked.cuh"
 
 using namespace pamm;
 
@@ -292,9 +292,10 @@ pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pam
         g_launches += 1;
         return s;
     }
-    if (weight_grad_mma_supported(k, n, m)) {
+    if (weight_grad_chunked_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_mma(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
+        const pamm_status s = launch_weight_grad_chunked(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped,
+                                                         accumulate);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;

@@ -22,7 +22,7 @@
 #pragma once
 #include "pamm_common.cuh"
 #include "sm100_ptx.cuh"
-#include "weight_grad_mma.cuh"
+#include "weight_grad_common.cuh"
 
 namespace pamm {
 
