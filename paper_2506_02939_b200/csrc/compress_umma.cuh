@@ -8,7 +8,8 @@
 //              the hidden dimension per pipeline stage, 128-byte swizzle
 //   warp 1     issues tcgen05.mma (M = 128 rows, N = generators of the chunk,
 //              K = 16 per instruction), fp32 accumulators in TMEM, two buffers
-//   warps 2-5  epilogue: each thread owns one row (TMEM lane), reads its scores
+//   warps 2-   epilogue, four warps per row tile of the super tile: each thread owns one
+//              row (TMEM lane) of one tile, reads its scores
 //              with tcgen05.ld and scans them in ascending j with a strict '>'
 //              so the lowest index wins ties; the epilogue of one tile overlaps
 //              the MMAs of the next
@@ -27,8 +28,8 @@
 
 namespace pamm {
 
-constexpr int CU_THREADS = 192;
-constexpr int CU_THREADS_EPS(int mt) { return 192 + mt * 128; }   // + one thread per row of the super tile for ||X_i||^2
+__host__ __device__ constexpr int CU_THREADS(int mt) { return 64 + mt * 128; }         // producer, MMA issuer, one epilogue thread per row of the super tile
+__host__ __device__ constexpr int CU_THREADS_EPS(int mt) { return 64 + mt * 256; }     // + one thread per row for ||X_i||^2
 constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
 constexpr int CU_TILE_M = 128;
 #ifndef PAMM_CU_BOX_ROWS
@@ -119,7 +120,7 @@ __host__ __device__ inline float neighbourhood_slack(int64_t n) { return 2.f * (
 // EPS = false: the paper's setting (epsilon = infinity), nothing is dropped.
 // EPS = true : eps2 = epsilon^2 and slack as above; *dropped counts the dropped rows.
 template <int MT, bool EPS>
-__global__ void __launch_bounds__(EPS ? CU_THREADS_EPS(MT) : CU_THREADS, 1)
+__global__ void __launch_bounds__(EPS ? CU_THREADS_EPS(MT) : CU_THREADS(MT), 1)
 compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
                      int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
                      int tmem_cols, int tmem_bufs, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
@@ -148,9 +149,9 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         for (int s = 0; s < stages; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&s_empty[s], EPS ? 1 + 4 * MT : 1); }
         for (int u = 0; u < 2; ++u) {
             ptx::mbar_init(&s_tfull[u], 1);
-            ptx::mbar_init(&s_tempty[u], 4);
+            ptx::mbar_init(&s_tempty[u], 4 * MT);
             ptx::mbar_init(&s_nfull[u], 4 * MT);
-            ptx::mbar_init(&s_nempty[u], 4);
+            ptx::mbar_init(&s_nempty[u], 4 * MT);
         }
         s_abort = 0;
         ptx::fence_barrier_init();
@@ -264,9 +265,10 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             }
             if (!ok) raise_status(DEV_TIMEOUT);
         }
-    } else if (EPS && warp >= 6) {
+    } else if (EPS && warp >= 2 + 4 * MT) {
         // ---------------- squared row norms: one row of the super tile per thread ----------------
-        const int my_mt = (threadIdx.x - 192) / CU_TILE_M, row_in_tile = (threadIdx.x - 192) % CU_TILE_M;
+        const int nt = threadIdx.x - CU_THREADS(MT);
+        const int my_mt = nt / CU_TILE_M, row_in_tile = nt % CU_TILE_M;
         const int ksteps_all = num_chunks * ksteps;
         uint32_t it = 0, sup = 0;
         bool ok = true;
@@ -307,32 +309,29 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         }
         if (!ok && lane == 0) raise_status(DEV_TIMEOUT);
     } else {
-        // ---------------- epilogue: one row per thread ----------------
+        // ---------------- epilogue: one row of one tile per thread ----------------
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
+        const int mt = (warp - 2) >> 2;                  // my row tile of the super tile
         const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
         if (x_is_ready) grid_dependency_wait();
-        for (int j = threadIdx.x - 64; j < kpad; j += 128) s_inv[j] = j < k ? c_invnorm[j] : 0.f;
-        for (int j = threadIdx.x - 64; j < k; j += 128) s_inv2[j] = c_invnorm[k + j];
-        ptx::named_barrier(1, 128);                      // the four epilogue warps share the norms
+        for (int j = threadIdx.x - 64; j < kpad; j += 128 * MT) s_inv[j] = j < k ? c_invnorm[j] : 0.f;
+        for (int j = threadIdx.x - 64; j < k; j += 128 * MT) s_inv2[j] = c_invnorm[k + j];
+        ptx::named_barrier(1, 128 * MT);                 // the epilogue warps share the norms
         uint32_t unit = 0, sup = 0;
         bool ok = true;
         for (int64_t st = r0; st < r1 && ok; st += super_rows, ++sup) {
-            float best[MT], s_best[MT];
-            int j_best[MT];
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) { best[mt] = -1.f; s_best[mt] = 0.f; j_best[mt] = 0; }
+            float best = -1.f, s_best = 0.f;
+            int j_best = 0;
+            const bool live = st + (int64_t)mt * CU_TILE_M < r1;
             for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
                 const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_tfull[buf], uph, abort_flag));   // warp-uniform
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t d_base = tmem_base + buf * (uint32_t)(MT * n_chunk) + lane_base;
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    if (st + (int64_t)mt * CU_TILE_M >= r1) continue;
+                if (live) {
                     // two register buffers: the TMEM load of the next 16 columns is in flight
                     // while the current 16 go through the tournament
-                    const uint32_t t_base = d_base + (uint32_t)(mt * n_chunk);
+                    const uint32_t t_base = tmem_base + buf * (uint32_t)(MT * n_chunk) + lane_base + (uint32_t)(mt * n_chunk);
                     const int jb = ch * n_chunk;
                     uint32_t va[16], vb[16];
                     ptx::tmem_ld_16cols(t_base, va);
@@ -340,11 +339,11 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                         ptx::tmem_ld_wait(va);
                         const bool second = c0 + 16 < n_chunk;
                         if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
-                        argmax16(va, s_inv + jb + c0, jb + c0, best[mt], s_best[mt], j_best[mt]);
+                        argmax16(va, s_inv + jb + c0, jb + c0, best, s_best, j_best);
                         if (second) {
                             ptx::tmem_ld_wait(vb);
                             if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
-                            argmax16(vb, s_inv + jb + c0 + 16, jb + c0 + 16, best[mt], s_best[mt], j_best[mt]);
+                            argmax16(vb, s_inv + jb + c0 + 16, jb + c0 + 16, best, s_best, j_best);
                         }
                     }
                 }
@@ -355,19 +354,16 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             if (ok && EPS) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_nfull[sup & 1u], (sup >> 1) & 1u, abort_flag));
             if (ok) {
                 int ndrop = 0;
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt) {
-                    const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
-                    if (row < r1) {
-                        float a = s_best[mt] * s_inv2[j_best[mt]];
-                        if (EPS) {     // Eq. 2: ||X_i - alpha C_f||^2 = ||X_i||^2 - S^2/||C_f||^2 against eps^2 ||X_i||^2
-                            const float nx = s_norm[sup & 1u][mt * CU_TILE_M + quad * 32 + lane];
-                            const float dist2 = nx - s_best[mt] * a;
-                            if (dist2 > (eps2 + slack) * nx) { a = 0.f; ++ndrop; }
-                        }
-                        f[row] = j_best[mt];
-                        alpha[row] = a;
+                const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
+                if (row < r1) {
+                    float a = s_best * s_inv2[j_best];
+                    if (EPS) {     // Eq. 2: ||X_i - alpha C_f||^2 = ||X_i||^2 - S^2/||C_f||^2 against eps^2 ||X_i||^2
+                        const float nx = s_norm[sup & 1u][mt * CU_TILE_M + quad * 32 + lane];
+                        const float dist2 = nx - s_best * a;
+                        if (dist2 > (eps2 + slack) * nx) { a = 0.f; ++ndrop; }
                     }
+                    f[row] = j_best;
+                    alpha[row] = a;
                 }
                 if (EPS) {
                     __syncwarp();
@@ -404,7 +400,7 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
         return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
-    cfg.blockDim = dim3(with_eps ? CU_THREADS_EPS(p.mt) : CU_THREADS);
+    cfg.blockDim = dim3(with_eps ? CU_THREADS_EPS(p.mt) : CU_THREADS(p.mt));
     cfg.dynamicSmemBytes = p.smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
