@@ -80,7 +80,7 @@ size_t pamm_workspace_bytes(pamm_ws_kind kind, int64_t b, int64_t n, int64_t m, 
 pamm_status pamm_draw_indices_host(int64_t b, int64_t k, uint64_t seed, int32_t* idx_out);
 
 /*
- * Step 1 -- choose generators (Algorithm 1: "Sample indices", "C <- A[I,:]",
+ * Step 1 -- choose generators (Algorithm 1, Compress: the index sampling, the gather of C,
  * and the norms eta_C of the generator rows).
  *   X        b x n, dtype dt, leading dimension ldx
  *   idx_in   NULL: draw I from `seed` as pamm_draw_indices_host does (ascending);
@@ -100,8 +100,8 @@ pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_
                                    void* stream);
 
 /*
- * Step 2 -- compress (Section 3.2 "Compressing A", Eq. 1, Lemma 1; Algorithm 1
- * lines "csim", "argmax", "alpha").  One streaming pass over X:
+ * Step 2 -- compress (Section 3.2 "Compressing A", Eq. 1, Lemma 1; Algorithm 1,
+ * Compress: cosine similarities, assignment, scales).  One streaming pass over X:
  *   S = X C^T;  f_i = the lowest j maximising |S_ij| / ||C_j||  (equivalently
  *   |csim(X_i, C_j)|, Lemma 1);  alpha_i = S_{i,f_i} / ||C_{f_i}||^2  (Eq. 1).
  * Products are exact, sums are accumulated in fp32.  A zero row gets f = 0,
@@ -114,7 +114,7 @@ pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm
                           int32_t* f, float* alpha, void* workspace, size_t ws_bytes, void* stream);
 
 /*
- * Steps 1+2 in one call (Algorithm 2, "C, alpha, f <- Compress(flatten(X), r)"):
+ * Steps 1+2 in one call (Algorithm 2: the Compress call on the flattened X):
  * draws I from `seed` (or uses idx_in), then compresses.  Arguments as above.
  */
 pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
@@ -124,7 +124,7 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
 
 /*
  * Step 3 -- contract (Section 3.2 "Approximate Matrix Multiplication";
- * Algorithm 1 ApproxMM: "B' <- alpha (.) B", "B~ <- index_add(B~, 0, f, B')"):
+ * Algorithm 1, ApproxMM: the alpha-scaling of B and the index_add into B~):
  *   B~[j,:] = sum over {i : f_i = j} of alpha_i * dY[i,:]      (k x m, fp32)
  * B' is never materialised.  dY is read once; rows are grouped by f with a
  * stable counting sort, summed in fp32 in ascending row order inside fixed-size
@@ -138,8 +138,8 @@ pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, 
                           float* Btilde, int64_t ldb, void* workspace, size_t ws_bytes, void* stream);
 
 /*
- * Step 4 -- weight gradient (Algorithm 1 ApproxMM, "O~ <- C^T B~"; Algorithm 3,
- * "grad W~ <- ApproxMM(C, alpha, f, grad Z)"):
+ * Step 4 -- weight gradient (Algorithm 1, ApproxMM: the final product; Algorithm 3,
+ * the weight gradient through ApproxMM):
  *   dW[r,c] = sum_j C[j,r] * B~[j,c]                          (n x m, fp32)
  *   C  k x n, dtype dt, ldc      Btilde  k x m fp32, ldb      dW  n x m fp32, ldw
  */
@@ -148,8 +148,8 @@ pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, p
                              float* dW, int64_t ldw, void* stream);
 
 /*
- * Step 2 with the neighbourhood condition (Section 3.2, Eq. 2; Algorithm 1 lines
- * "e = ||A - alpha (.) C[f,:]||" and "alpha[e > eps] <- 0").  As pamm_compress;
+ * Step 2 with the neighbourhood condition (Section 3.2, Eq. 2; Algorithm 1,
+ * Compress: the distance e and the masked assignment of alpha).  As pamm_compress;
  * in addition a row whose representative is farther than eps ||X_i|| is dropped,
  * i.e. gets alpha_i = 0 (f_i is still reported).  The test follows Eq. 2 (relative
  * to ||X_i||; Algorithm 1 prints it without the norm).  It is evaluated in fp32 as

@@ -54,7 +54,7 @@ static double widen(const void *base, int dtype, int64_t idx)
     }
 }
 
-/* Algorithm 1, "C <- A[I,:]" and the squared row norms of C.
+/* Algorithm 1, Compress: the gather C = A[I,:] and the squared row norms of C.
  * C_out is k x n doubles, q_out[j] = sum_l C_jl^2. */
 int pamm_oracle_gather(const void *A, int dtype, int64_t b, int64_t n, int64_t lda,
                        const int32_t *I, int64_t k, double *C_out, double *q_out)
@@ -168,7 +168,7 @@ double pamm_oracle_beta(int64_t b, int64_t eta)
 }
 
 /* Algorithm 1 "ApproxMM", first two steps: B' = alpha (.) B and
- * B~ <- index_add(B~, 0, f, B'), i.e. B~[j,:] = sum_{i: f_i = j} alpha_i B_i
+ * the index_add of B' into B~ keyed by f, i.e. B~[j,:] = sum_{i: f_i = j} alpha_i B_i
  * (Section 3.2, "Approximate Matrix Multiplication"). Rows visited in
  * ascending i. Bt_out is k x m doubles. */
 int pamm_oracle_contract(const int32_t *f, const double *alpha, const void *B, int dtype,

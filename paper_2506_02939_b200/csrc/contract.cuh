@@ -1,5 +1,5 @@
 // Step 3: B~[j,:] = sum_{i: f_i = j} alpha_i * dY[i,:]  (Algorithm 1 ApproxMM,
-// "B' <- alpha (.) B" and "index_add"), as a deterministic segmented reduction.
+// the alpha-scaling of B and the index_add), as a deterministic segmented reduction.
 //
 //   hist    : per block of SORT_BLK rows, a histogram of f            (integers)
 //   scan    : exclusive scans -> segment starts and per-block offsets

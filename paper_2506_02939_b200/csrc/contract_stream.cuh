@@ -1,4 +1,4 @@
-// Step 3, main pass (Algorithm 1 ApproxMM: "B' <- alpha (.) B", "index_add"):
+// Step 3, main pass (Algorithm 1, ApproxMM: alpha-scaling of B and index_add):
 // B~[j,:] = sum_{i: f_i = j} alpha_i * dY[i,:] over the rows sorted by f, with the
 // rows of dY staged through shared memory by bulk asynchronous copies.
 //

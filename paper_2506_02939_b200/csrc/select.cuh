@@ -1,4 +1,4 @@
-// Step 1: generator selection (Algorithm 1: "Sample indices I", "C <- A[I,:]",
+// Step 1: generator selection (Algorithm 1, Compress: index sampling, the gather of C,
 // and the norms of the generator rows).  One launch, no cross-CTA dependency:
 // every CTA recomputes the k candidate indices in shared memory, ranks its own
 // candidate (rank = sorted position), copies that row of X into C with one

@@ -1,5 +1,5 @@
 // Step 4 on tensor cores for k > 128 (bf16 generators): dW = C^T B~ (Algorithm 1
-// ApproxMM, "O~ <- C^T B~"), persistent and pipelined over chunks of 64 generators.
+// ApproxMM, the final product), persistent and pipelined over chunks of 64 generators.
 //
 // One CTA per SM takes a contiguous run of 128 x 128 output tiles (numbered column
 // block by column block, so neighbours share their B~ columns in L2).  Every tile

@@ -1,5 +1,5 @@
 // Step 4 on tensor cores for k <= 128 (bf16 generators): dW = C^T B~ (Algorithm 1
-// ApproxMM, "O~ <- C^T B~") as a persistent, pipelined kernel.
+// ApproxMM, the final product) as a persistent, pipelined kernel.
 //
 // The product is bound by writing dW (2k flops per 4 bytes written), so the
 // kernel is built around keeping stores in flight.  One CTA per SM takes a

@@ -1,5 +1,5 @@
 // Step 4 on CUDA cores: dW[r,c] = sum_j C[j,r] * B~[j,c]  (Algorithm 1 ApproxMM,
-// "O~ <- C^T B~").  Each thread owns four consecutive columns of one output
+// the final product).  Each thread owns four consecutive columns of one output
 // row and walks the k generators in ascending order with fp32 FMAs.  Used for
 // fp32 generators and whenever the tensor-core path does not apply.
 #pragma once
