@@ -34,7 +34,7 @@ PROF_EVERY = 16     # one step in PROF_EVERY carries per-kernel CUDA events, ano
                     # the rest run event-free, since an event between two kernels serialises their launches
 # DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
 # summarised under profiles/, keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {"c4": 811204096}     # contract_stream_kernel<bf16,2,1>: 806.14 MB read + 5.06 MB written
+NCU_TRAFFIC_BYTES = {"c4": 811101696}     # contract_stream_kernel<bf16,2,1>: 806.12 MB read + 4.98 MB written
 
 
 def env_int(name, default):
@@ -497,7 +497,7 @@ def run_layer_loop(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 2000; 20 for --impl reference)")
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 3000; 20 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=None, help="untimed steps (default 20; 2 for --impl reference)")
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="c4", help="c1..c5; c4 (LLaMA-1B-shaped) is the headline configuration")
@@ -513,7 +513,7 @@ def main():
     ap.add_argument("--distinct-layers", type=int, default=4, help="distinct synthetic input sets in the --layers mode")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 2000 if args.impl == "cuda" else 20
+        args.steps = 3000 if args.impl == "cuda" else 20
     if args.warmup is None:
         args.warmup = 20 if args.impl == "cuda" else 2
     if args.impl == "cuda":
