@@ -396,8 +396,7 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
         return PAMM_ERR_CUDA;
     auto kern = with_eps ? (p.mt == 2 ? compress_umma_kernel<2, true> : compress_umma_kernel<1, true>)
                          : (p.mt == 2 ? compress_umma_kernel<2, false> : compress_umma_kernel<1, false>);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
-        return PAMM_ERR_CUDA;
+    if (!ensure_dynamic_smem((const void*)kern, p.smem_bytes)) return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
     cfg.blockDim = dim3(with_eps ? CU_THREADS_EPS(p.mt) : CU_THREADS(p.mt));

@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "../../include/pamm.h"
@@ -138,5 +139,10 @@ __host__ __device__ inline uint32_t perm_apply(const PermKey& pk, uint32_t x) {
 }
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Raises a kernel's dynamic shared-memory limit when a launch needs more than the
+// 48 KiB default, remembering per device and kernel what has been granted already
+// so that the driver call is not repeated on every launch.
+bool ensure_dynamic_smem(const void* kernel, size_t bytes);
 
 }  // namespace pamm

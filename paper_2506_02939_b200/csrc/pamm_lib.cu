@@ -4,7 +4,9 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "pamm_common.cuh"
@@ -18,6 +20,22 @@
 #include "weight_grad_chunked.cuh"
 
 using namespace pamm;
+
+namespace pamm {
+bool ensure_dynamic_smem(const void* kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return true;
+    static std::mutex mu;
+    static std::map<std::pair<int, const void*>, size_t> granted;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    size_t& have = granted[{dev, kernel}];
+    if (have >= bytes) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+    have = bytes;
+    return true;
+}
+}  // namespace pamm
 
 namespace {
 
@@ -91,9 +109,7 @@ pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int6
                           const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
                           cudaStream_t st) {
     const size_t smem = (size_t)k * 4;
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(select_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return PAMM_ERR_CUDA;
+    if (!ensure_dynamic_smem((const void*)select_kernel<T>, smem)) return PAMM_ERR_CUDA;
     const PermKey pk = make_perm_key(seed, (uint32_t)b);
     const int grid = (int)k;
     launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, true, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
@@ -146,9 +162,9 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
                             int64_t k, float* Bt, int64_t ldb, const ContractWs& w, cudaStream_t st) {
     constexpr int V = Vec16<T>::N;
     const size_t hsmem = (size_t)k * 4;
-    if (hsmem > 48 * 1024 &&
-        (cudaFuncSetAttribute(contract_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess ||
-         cudaFuncSetAttribute(contract_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hsmem) != cudaSuccess))
+    if (!ensure_dynamic_smem((const void*)contract_hist_kernel, hsmem) ||
+        !ensure_dynamic_smem((const void*)contract_scatter_kernel, hsmem) ||
+        !ensure_dynamic_smem((const void*)contract_scan_scatter_kernel, hsmem))
         return PAMM_ERR_CUDA;
     launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k, w.hist);
     if (w.nb * w.nb * k <= FUSED_SCAN_LIMIT) {
@@ -170,8 +186,7 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
                     : p.rps == 4 ? contract_stream_kernel<T, 1, 4>
                     : p.rps == 2 ? contract_stream_kernel<T, 1, 2>
                                  : contract_stream_kernel<T, 1, 1>;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes) != cudaSuccess)
-            return PAMM_ERR_CUDA;
+        if (!ensure_dynamic_smem((const void*)kern, p.smem_bytes)) return PAMM_ERR_CUDA;
         prof_begin(PAMM_PROF_CONTRACT, st);
         launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, alpha, (const T*)dY, ldy, m,
                (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots, p.row_pitch,

@@ -266,8 +266,7 @@ inline pamm_status launch_weight_grad_chunked(const void* C, int64_t ldc, int64_
     const int64_t total = (int64_t)n_tiles * m_tiles;
     if (total * nch >= (1ll << 31)) return PAMM_ERR_UNSUPPORTED;
     const size_t smem = 1024 + (size_t)WC_STAGES * WC_STAGE_BYTES + 2 * WP_OUT_HALF_BYTES;
-    if (cudaFuncSetAttribute(weight_grad_chunked_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return PAMM_ERR_CUDA;
+    if (!ensure_dynamic_smem((const void*)weight_grad_chunked_kernel, smem)) return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)std::min<int64_t>(total, sms));
     cfg.blockDim = dim3(WC_THREADS);

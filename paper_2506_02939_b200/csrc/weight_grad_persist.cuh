@@ -294,8 +294,7 @@ inline pamm_status launch_weight_grad_persist(const void* C, int64_t ldc, int64_
         parts = std::max(1, std::min(n_tiles, sms / m_tiles));
         grid = (int64_t)m_tiles * parts;
     }
-    if (cudaFuncSetAttribute(weight_grad_persist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return PAMM_ERR_CUDA;
+    if (!ensure_dynamic_smem((const void*)weight_grad_persist_kernel, smem)) return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(WP_THREADS);

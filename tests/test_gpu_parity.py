@@ -279,3 +279,16 @@ def test_weight_grad_accumulate_adds_to_dW(k, n, m, dtype):
     pamm.weight_grad_accumulate(C, Bt, dW)
     assert torch.allclose(dW, base + 2 * once, rtol=1e-6, atol=1e-5)
     assert pamm.last_device_status() == pamm.OK
+
+
+def test_contract_with_many_generators_uses_large_shared_histograms():
+    # k = 13000: the per-block histograms of the sort need more than the default 48 KiB of shared memory
+    rng = np.random.default_rng(61)
+    b, m, k = 20000, 72, 13000
+    _, dY = synth.random_case(b, 8, m, "bf16", seed=62)
+    f = rng.integers(0, k, size=b).astype(np.int32)
+    a = rng.standard_normal(b).astype(np.float32)
+    Bt = pamm.contract(torch.from_numpy(f).cuda(), torch.from_numpy(a).cuda(), parity.to_device(dY), k)
+    assert pamm.last_device_status() == pamm.OK
+    ref = orc.contract(f, a.astype(np.float64), dY, k)
+    assert parity.rel_fro(Bt.cpu().numpy(), ref) <= 1e-5
