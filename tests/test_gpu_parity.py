@@ -131,8 +131,9 @@ def test_results_are_bit_reproducible():
                                b_.view(torch.uint8) if b_.dtype == torch.bfloat16 else b_)
 
 
-def test_outputs_stay_inside_their_buffers():
-    b, n, m, k = 1500, 136, 264, 24
+@pytest.mark.parametrize("b,n,m,k", [(1500, 136, 264, 24), (1300, 200, 392, 200), (2100, 72, 3080, 300)])
+def test_outputs_stay_inside_their_buffers(b, n, m, k):
+    # guard regions around every output and the workspace: k <= 128 and k > 128 products, one and two rows per ring slot
     X, dY = synth.random_case(b, n, m, "bf16", seed=9, centres=10)
     Xd, dYd = parity.to_device(X), parity.to_device(dY)
     G = 64
