@@ -182,6 +182,19 @@ contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, co
     __shared__ int32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int me = blockIdx.x;
+    // f is older than the histogram kernel, which did not let this kernel in before its
+    // own wait for f's producer had returned: the keys can be fetched and ranked inside
+    // their warp before this kernel waits for the histograms.
+    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
+    int32_t key = -1;
+    if (i < b) {
+        key = f[i];
+        if (key < 0 || key >= k) key = -1;
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, key);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    const int leader = __ffs(peers) - 1;
+    const int count = __popc(peers);
     grid_dependency_wait();
     grid_launch_dependents();
     if (tid == 0) s_carry = 0;
@@ -196,14 +209,15 @@ contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, co
         if (jj < width) {
             const int32_t* col = hist + j0 + jj;
             int blk = grp;
-            for (; blk + 3 * groups < nb; blk += 4 * groups) {   // four independent loads in flight
-                const int32_t c0 = __ldg(col + (int64_t)blk * k);
-                const int32_t c1 = __ldg(col + (int64_t)(blk + groups) * k);
-                const int32_t c2 = __ldg(col + (int64_t)(blk + 2 * groups) * k);
-                const int32_t c3 = __ldg(col + (int64_t)(blk + 3 * groups) * k);
-                total += (c0 + c1) + (c2 + c3);
-                before += (blk < me ? c0 : 0) + (blk + groups < me ? c1 : 0) + (blk + 2 * groups < me ? c2 : 0) +
-                          (blk + 3 * groups < me ? c3 : 0);
+            for (; blk + 7 * groups < nb; blk += 8 * groups) {   // eight independent loads in flight
+                int32_t c[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) c[u] = __ldg(col + (int64_t)(blk + u * groups) * k);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    total += c[u];
+                    before += blk + u * groups < me ? c[u] : 0;
+                }
             }
             for (; blk < nb; blk += groups) {
                 const int32_t c = __ldg(col + (int64_t)blk * k);
@@ -253,26 +267,16 @@ contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, co
     }
     if (me == 0 && tid == 0) seg_start[k] = s_carry;
 
-    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
-    int32_t j = -1;
-    if (i < b) {
-        j = f[i];
-        if (j < 0 || j >= k) j = -1;
-    }
-    const unsigned peers = __match_any_sync(0xffffffffu, j);
-    const int rank = __popc(peers & ((1u << lane) - 1u));
-    const int leader = __ffs(peers) - 1;
-    const int count = __popc(peers);
     for (int w = 0; w < SORT_BLK / 32; ++w) {
         __syncthreads();
         if (warp == w) {
             int32_t base = 0;
-            if (lane == leader && j >= 0) {
-                base = s_next[j];
-                s_next[j] = base + count;
+            if (lane == leader && key >= 0) {
+                base = s_next[key];
+                s_next[key] = base + count;
             }
             base = __shfl_sync(0xffffffffu, base, leader);
-            if (j >= 0) perm[base + rank] = (int32_t)i;
+            if (key >= 0) perm[base + rank] = (int32_t)i;
         }
     }
 }
