@@ -272,6 +272,15 @@ typedef enum { PAMM_PROF_COMPRESS = 0, PAMM_PROF_CONTRACT = 1, PAMM_PROF_WEIGHT_
 unsigned long long pamm_launch_count(void);
 pamm_status pamm_set_profile_events(pamm_prof_kind kind, void* start_event, void* stop_event);
 
+/*
+ * Self-test of the failure path (no counterpart in the paper): launches one small
+ * kernel that waits, with the library's bounded wait and a limit of 2048 polls, on a
+ * barrier nothing completes.  The wait gives up, the kernel ends normally, and
+ * pamm_last_device_status(stream) then reports PAMM_ERR_TIMEOUT once; the context
+ * stays usable.  Nothing faults, traps or spins without a limit.
+ */
+pamm_status pamm_selftest_bounded_wait(void* stream);
+
 /* Library version as major*10000 + minor*100 + patch. */
 int pamm_version(void);
 

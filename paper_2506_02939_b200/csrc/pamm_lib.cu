@@ -320,7 +320,29 @@ pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pam
 
 }  // namespace
 
+// One CTA waits, with the library's bounded wait and a short limit, on a barrier that
+// nothing will ever complete; the wait must give up, raise the status word and let the
+// kernel end normally.
+__global__ void selftest_bounded_wait_kernel(uint32_t polls) {
+    __shared__ uint64_t s_bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&s_bar, 1);
+        s_abort = 0;
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = &s_abort;
+    const bool done = ptx::mbar_wait(&s_bar, 0, abort_flag, polls);
+    if (!done && (threadIdx.x & 31) == 0) raise_status(DEV_TIMEOUT);
+}
+
 extern "C" {
+
+pamm_status pamm_selftest_bounded_wait(void* stream) {
+    launch(selftest_bounded_wait_kernel, dim3(1), dim3(64), 0, (cudaStream_t)stream, false, (uint32_t)2048);
+    return launch_status();
+}
 
 const char* pamm_status_string(pamm_status s) {
     switch (s) {

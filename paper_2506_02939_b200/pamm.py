@@ -44,6 +44,7 @@ _SIGNATURES = {
     "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
     "pamm_last_device_status": ([_vp], _ci),
+    "pamm_selftest_bounded_wait": ([_vp], _ci),
     "pamm_launch_count": ([], ctypes.c_ulonglong),
     "pamm_set_profile_events": ([_ci, _vp, _vp], _ci),
 }
@@ -247,6 +248,11 @@ def qkv_step_host(X_host, dY_host, k: int, seed: int, dW_host, arena, f_host=Non
                                    _ptr(f_host), _ptr(alpha_host), _ptr(arena), arena.numel(), _stream(stream)),
            "pamm_qkv_step_host")
     return dW_host
+
+
+def selftest_bounded_wait(stream=None) -> None:
+    """Launch the kernel whose bounded wait must run out (sets ERR_TIMEOUT in the device status word)."""
+    _check(_lib.pamm_selftest_bounded_wait(_stream(stream)), "pamm_selftest_bounded_wait")
 
 
 def last_device_status(stream=None) -> int:

@@ -293,3 +293,12 @@ def test_contract_with_many_generators_uses_large_shared_histograms():
     assert pamm.last_device_status() == pamm.OK
     ref = orc.contract(f, a.astype(np.float64), dY, k)
     assert parity.rel_fro(Bt.cpu().numpy(), ref) <= 1e-5
+
+
+def test_a_wait_that_runs_out_reports_a_timeout_and_the_context_lives_on():
+    assert pamm.last_device_status() == pamm.OK
+    pamm.selftest_bounded_wait()                                   # waits on a barrier nothing completes, with a limit
+    assert pamm.last_device_status() == pamm.ERR_TIMEOUT
+    assert pamm.last_device_status() == pamm.OK
+    X, dY = synth.random_case(600, 72, 40, "bf16", seed=71, centres=5, dy_scale=1e-3)
+    parity.run_and_compare(X, dY, 20, seed=72)                     # the library still works afterwards
