@@ -302,3 +302,36 @@ def test_a_wait_that_runs_out_reports_a_timeout_and_the_context_lives_on():
     assert pamm.last_device_status() == pamm.OK
     X, dY = synth.random_case(600, 72, 40, "bf16", seed=71, centres=5, dy_scale=1e-3)
     parity.run_and_compare(X, dY, 20, seed=72)                     # the library still works afterwards
+
+
+def test_a_whole_step_can_be_captured_in_a_cuda_graph():
+    # launch-bound sizes profit from replaying the seven launches of a step as one graph
+    X, dY = synth.random_case(2048, 512, 1536, "f32", seed=81, centres=16, dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    k = 4
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, 3)
+    Bt = pamm.alloc_matrix(k, 1536, torch.float32)
+    dW = pamm.alloc_matrix(512, 1536, torch.float32)
+    ws = pamm.alloc_workspace(pamm.WS_CONTRACT, 2048, 512, 1536, k, pamm.F32)
+
+    def step(stream=None):
+        pamm.compress_fused(Xd, k, 3, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+        pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+
+    step()
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (f, alpha, Bt, dW)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step(torch.cuda.current_stream())
+    for t in (f, alpha, Bt, dW):
+        t.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert pamm.last_device_status() == pamm.OK
+    for got, ref in zip((f, alpha, Bt, dW), want):
+        assert torch.equal(got, ref)
