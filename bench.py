@@ -30,11 +30,11 @@ if str(ROOT) not in sys.path:
 METRIC = "PAMM compress + weight-grad tokens/sec per QKV layer; achieved HBM GB/s vs peak"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0      # sustained, inside a long step
+NOMINAL_HBM_GBS = 8000.0           # the data-sheet figure the fractions "of nominal" refer to
 PROF_EVERY = 16     # one step in PROF_EVERY carries per-kernel CUDA events, another one the stage events;
                     # the rest run event-free, since an event between two kernels serialises their launches
-# DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture
-# summarised under profiles/, keyed by workload; None until captured.
-NCU_TRAFFIC_BYTES = {"c4": 811101696}     # contract_stream_kernel<bf16,2,1>: 806.12 MB read + 4.98 MB written
+MIN_SAMPLES = 32    # stage / kernel samples behind every reported median; short runs top up after the timed region
+TRAFFIC_FILE = ROOT / "profiles" / "dominant_kernel_traffic.txt"
 
 
 def env_int(name, default):
@@ -131,12 +131,33 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
-def algorithmic_bytes(b, n, m, k, e):
+def ncu_traffic(workload: str, kernel_source: Path):
+    """DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised under
+    profiles/.  A line of the file reads `workload bytes sha256-of-the-kernel-source ...`; the figure is
+    reported only while the kernel's source is the one the counters were taken from."""
+    import hashlib
+    try:
+        digest = hashlib.sha256(kernel_source.read_bytes()).hexdigest()[:16]
+        for line in TRAFFIC_FILE.read_text().splitlines():
+            p = line.split()
+            if len(p) >= 3 and not line.startswith("#") and p[0] == workload and p[2] == digest:
+                return int(p[1])
+    except (OSError, ValueError):
+        pass
+    return None
+
+
+def stats(x) -> dict:
+    x = np.asarray(x, dtype=np.float64)
+    return {"count": int(x.size), "median": float(np.median(x)), "min": float(x.min()), "mean": float(x.mean())}
+
+
+def algorithmic_bytes(b, n, m, k, e, dw_e=4):
     """Bytes the method itself must move per step (per layer), by stage."""
     return {
         "compress": b * n * e + 8 * b + k * n * e,
         "contract": b * m * e + 8 * b,
-        "weight_grad": n * m * 4 + k * n * e + k * m * 4,
+        "weight_grad": n * m * dw_e + k * n * e + k * m * 4,
     }
 
 
@@ -225,8 +246,11 @@ def run_cuda(args):
     f = torch.empty(b, dtype=torch.int32, device=dev)
     alpha = torch.empty(b, dtype=torch.float32, device=dev)
     Bt = torch.empty((k, m), dtype=torch.float32, device=dev)
-    dW = torch.empty((n, m), dtype=torch.float32, device=dev)
+    dw_tdt = torch.bfloat16 if args.dw_dtype == "bf16" else torch.float32
+    layout = pamm.DW_MN if args.layout == "mn" else pamm.DW_NM
+    dW = torch.empty((m, n) if layout == pamm.DW_MN else (n, m), dtype=dw_tdt, device=dev)
     ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, dt_code, dev)
+    sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, dt_code, dev)     # the forward's counts of f, for the backward's sort
     stream = torch.cuda.current_stream()
 
     eps = args.eps
@@ -234,17 +258,18 @@ def run_cuda(args):
 
     def forward(seed):
         if eps is None:
-            pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, stream=stream)
+            pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, sort_products=sp, stream=stream)
         else:     # neighbourhood condition (Eq. 2): select, then compress with the row-norm warps
             pamm.select_generators(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, stream=stream)
-            pamm.compress_eps(X, C, invn, eps, f=f, alpha=alpha, dropped=dropped, stream=stream)
+            pamm.compress_eps(X, C, invn, eps, f=f, alpha=alpha, dropped=dropped, sort_products=sp, stream=stream)
 
     def backward():
         if eps is None:
-            pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, workspace=ws, stream=stream)
+            pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, layout=layout, sort_products=sp, workspace=ws,
+                                      stream=stream)
         else:     # beta = b / (b - eta) applied by the product's epilogue (Eq. 4-5)
-            pamm.contract(f, alpha, dY, k, Btilde=Bt, workspace=ws, stream=stream)
-            pamm.weight_grad_beta(C, Bt, b, dropped, dW=dW, stream=stream)
+            pamm.contract(f, alpha, dY, k, Btilde=Bt, sort_products=sp, workspace=ws, stream=stream)
+            pamm.weight_grad_beta(C, Bt, b, dropped, dW=dW, layout=layout, stream=stream)
 
     def step(seed):
         forward(seed)
@@ -259,16 +284,36 @@ def run_cuda(args):
 
     # ---- timed region: device-resident inputs ----------------------------------
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    # per-kernel event pairs on every PROF_EVERY-th step only: an event between two
-    # kernels serialises them, the other steps keep the back-to-back launch overlap
-    prof_steps = [s for s in range(K) if s % PROF_EVERY == 0]
-    kev = {kind: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in prof_steps]
-           for kind in (pamm.PROF_COMPRESS, pamm.PROF_CONTRACT, pamm.PROF_WEIGHT_GRAD)}
-    for kind in kev:                       # create the underlying CUDA events
-        for a, z in kev[kind]:
-            a.record(stream)
-            z.record(stream)
+    KINDS = (pamm.PROF_COMPRESS, pamm.PROF_CONTRACT, pamm.PROF_WEIGHT_GRAD)
+
+    def new_event():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)          # creates the underlying CUDA event, whose handle the library records later
+        return e
+
+    def kernel_step(seed):
+        """One step with an event pair around each step's main kernel."""
+        pairs = {kind: (new_event(), new_event()) for kind in KINDS}
+        for kind in KINDS:
+            pamm.set_profile_events(kind, *pairs[kind])
+        step(seed)
+        for kind in KINDS:
+            pamm.set_profile_events(kind, None, None)
+        return pairs
+
+    def staged_step(seed):
+        """One step with events around the forward and the backward stage."""
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        forward(seed)
+        e[1].record(stream)
+        backward()
+        e[2].record(stream)
+        return e
+
+    # event pairs on a few steps only: an event between two kernels serialises them,
+    # the other steps keep the back-to-back launch overlap
+    kernel_samples, stage_samples = [], []
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
     launches0 = pamm.launch_count()
@@ -277,31 +322,30 @@ def run_cuda(args):
     sampler.start()
     t_begin.record(stream)
     for s in range(K):
-        if s % PROF_EVERY == 0:
-            for kind in kev:
-                pamm.set_profile_events(kind, kev[kind][s // PROF_EVERY][0], kev[kind][s // PROF_EVERY][1])
-        elif s % PROF_EVERY == 1:
-            for kind in kev:
-                pamm.set_profile_events(kind, None, None)
-        staged = K < PROF_EVERY or s % PROF_EVERY == PROF_EVERY // 2
-        if staged:
-            ev[s][0].record(stream)
-        forward(w.index_seed + s)
-        if staged:
-            ev[s][1].record(stream)
-        backward()
-        if staged:
-            ev[s][2].record(stream)
+        if s % PROF_EVERY == 0 and K >= PROF_EVERY:
+            kernel_samples.append(kernel_step(w.index_seed + s))
+        elif s % PROF_EVERY == PROF_EVERY // 2 and K >= PROF_EVERY:
+            stage_samples.append(staged_step(w.index_seed + s))
+        else:
+            step(w.index_seed + s)
     t_end.record(stream)
     torch.cuda.synchronize()
     launches = pamm.launch_count() - launches0
     barrier()
+    in_region = (len(kernel_samples), len(stage_samples))
+    # a short run yields too few samples for a median: top them up in an untimed pass over the same steps
+    extra = 0
+    while len(kernel_samples) < MIN_SAMPLES or len(stage_samples) < MIN_SAMPLES:
+        kernel_samples.append(kernel_step(w.index_seed + extra))
+        step(w.index_seed + extra)
+        stage_samples.append(staged_step(w.index_seed + extra))
+        step(w.index_seed + extra)
+        extra += 1
+    torch.cuda.synchronize()
     covers = "timed region"
     if t_begin.elapsed_time(t_end) < 500.0:
         # a region this short yields too few 50 ms samples: keep sampling over an untimed repeat of the same steps
         covers = "timed region + untimed repeat of it (region shorter than 0.5 s)"
-        for kind in kev:
-            pamm.set_profile_events(kind, None, None)
         t_rep = time.perf_counter()
         while time.perf_counter() - t_rep < 0.5:
             for s in range(16):
@@ -309,17 +353,16 @@ def run_cuda(args):
             torch.cuda.synchronize()
     clocks = sampler.stop()
     clocks["covers"] = covers
-    for kind in kev:
-        pamm.set_profile_events(kind, None, None)
     status = pamm.last_device_status()
     if status != pamm.OK:
         raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
     ms_total_local = t_begin.elapsed_time(t_end)
     ms_total, tokens = aggregate(ms_total_local, b * K, device=dev)
-    plain = [s for s in range(K) if K < PROF_EVERY or s % PROF_EVERY == PROF_EVERY // 2]
-    fwd = np.array([ev[s][0].elapsed_time(ev[s][1]) for s in plain])
-    bwd = np.array([ev[s][1].elapsed_time(ev[s][2]) for s in plain])
-    kern = {kind: np.array([a.elapsed_time(z) for a, z in kev[kind]]) for kind in kev}
+    fwd = np.array([e[0].elapsed_time(e[1]) for e in stage_samples])
+    bwd = np.array([e[1].elapsed_time(e[2]) for e in stage_samples])
+    kern = {kind: np.array([p[kind][0].elapsed_time(p[kind][1]) for p in kernel_samples]) for kind in KINDS}
+    sampling = {"kernel_events_in_timed_region": in_region[0], "stage_events_in_timed_region": in_region[1],
+                "added_in_untimed_pass_after_it": [len(kernel_samples) - in_region[0], len(stage_samples) - in_region[1]]}
 
     # ---- end to end through the host-buffer entry point ----------------------------
     arena = pamm.alloc_workspace(pamm.WS_STEP_HOST, b, n, m, k, dt_code, dev)
@@ -342,38 +385,53 @@ def run_cuda(args):
     if rank != 0:
         return
     peak, peak_tf, peak_kind = measured_peaks()
-    ab = algorithmic_bytes(b, n, m, k, e)
-    t_contract = float(kern[pamm.PROF_CONTRACT].mean()) * 1e-3
+    dw_e = 2 if args.dw_dtype == "bf16" else 4
+    ab = algorithmic_bytes(b, n, m, k, e, dw_e)
+    st_f, st_b = stats(fwd), stats(bwd)
+    st_k = {"compress": stats(kern[pamm.PROF_COMPRESS]), "contract_main": stats(kern[pamm.PROF_CONTRACT]),
+            "weight_grad": stats(kern[pamm.PROF_WEIGHT_GRAD])}
+    t_contract = st_k["contract_main"]["median"] * 1e-3
     achieved = ab["contract"] / t_contract / 1e9
+
+    def frac(gbs):
+        return {"gbs": gbs, "of_measured": gbs / peak, "of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
     stages = {
-        "compress_ms": float(np.median(fwd)), "contract_wgrad_ms": float(np.median(bwd)),
-        "compress_tokens_per_s": b / (float(np.median(fwd)) * 1e-3),
-        "contract_wgrad_tokens_per_s": b / (float(np.median(bwd)) * 1e-3),
-        "compress_stage_gbs": (ab["compress"]) / (float(np.median(fwd)) * 1e-3) / 1e9,
-        "contract_wgrad_stage_gbs": (ab["contract"] + ab["weight_grad"]) / (float(np.median(bwd)) * 1e-3) / 1e9,
-        "kernel_ms": {"compress": float(kern[pamm.PROF_COMPRESS].mean()), "contract_main": float(kern[pamm.PROF_CONTRACT].mean()),
-                      "weight_grad": float(kern[pamm.PROF_WEIGHT_GRAD].mean())},
-        "kernel_gbs": {"compress": ab["compress"] / (float(kern[pamm.PROF_COMPRESS].mean()) * 1e-3) / 1e9,
-                       "contract_main": achieved,
-                       "weight_grad": ab["weight_grad"] / (float(kern[pamm.PROF_WEIGHT_GRAD].mean()) * 1e-3) / 1e9},
+        "sampling": sampling,
+        "compress_ms": st_f, "contract_wgrad_ms": st_b,
+        "compress_tokens_per_s": b / (st_f["median"] * 1e-3),
+        "contract_wgrad_tokens_per_s": b / (st_b["median"] * 1e-3),
+        "compress_stage": frac(ab["compress"] / (st_f["median"] * 1e-3) / 1e9),
+        "compress_stage_best": frac(ab["compress"] / (st_f["min"] * 1e-3) / 1e9),
+        "contract_wgrad_stage": frac((ab["contract"] + ab["weight_grad"]) / (st_b["median"] * 1e-3) / 1e9),
+        "contract_wgrad_stage_best": frac((ab["contract"] + ab["weight_grad"]) / (st_b["min"] * 1e-3) / 1e9),
+        "whole_step": frac(sum(ab.values()) / (ms_total / K * 1e-3) / 1e9),
+        "kernel_ms": st_k,
+        "kernel": {"compress": frac(ab["compress"] / (st_k["compress"]["median"] * 1e-3) / 1e9),
+                   "contract_main": frac(achieved),
+                   "weight_grad": frac(ab["weight_grad"] / (st_k["weight_grad"]["median"] * 1e-3) / 1e9)},
+        "algorithmic_bytes": ab,
     }
-    stages["compress_stage_frac"] = stages["compress_stage_gbs"] / peak
-    stages["contract_wgrad_stage_frac"] = stages["contract_wgrad_stage_gbs"] / peak
+    stages["compress_stage_frac"] = stages["compress_stage"]["of_measured"]
+    stages["contract_wgrad_stage_frac"] = stages["contract_wgrad_stage"]["of_measured"]
     saved = pamm.saved_bytes(b, n, k, dt_code)
     # the dominant kernel: the contract main pass (HBM-bound), except where the scoring contraction is heavy enough to
     # make compress both the longest kernel and tensor-bound (2 b k n flops against b n e bytes: k above the ridge)
-    t_compress = float(kern[pamm.PROF_COMPRESS].mean()) * 1e-3
+    t_compress = st_k["compress"]["median"] * 1e-3
     flops = 2.0 * b * k * n
     if w.dtype == "bf16" and t_compress > t_contract and flops / ab["compress"] > peak_tf * 1e12 / (peak * 1e9):
         tf = flops / t_compress / 1e12
         roofline = {"bound": "tensor", "kernel": "compress_umma_kernel (scoring X C^T + argmax)", "achieved": tf, "peak": peak_tf,
                     "peak_source": f"of {peak_kind} (sustained bf16)", "unit": "TFLOP/s", "frac": tf / peak_tf, "traffic": None,
-                    "algorithmic_flops": flops}
+                    "algorithmic_flops": flops, "samples": st_k["compress"]["count"]}
     else:
         roofline = {"bound": "hbm", "kernel": "contract_stream_kernel (contract main pass)", "achieved": achieved, "peak": peak,
                     "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": NCU_TRAFFIC_BYTES.get(w.name) if k == w.ks[0] and args.eps is None else None,
-                    "algorithmic_bytes": ab["contract"]}
+                    "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                    "traffic": ncu_traffic(w.name, ROOT / "paper_2506_02939_b200" / "csrc" / "contract_stream.cuh")
+                    if k == w.ks[0] and args.eps is None else None,
+                    "algorithmic_bytes": ab["contract"], "samples": st_k["contract_main"]["count"],
+                    "achieved_best": ab["contract"] / (st_k["contract_main"]["min"] * 1e-3) / 1e9}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -396,7 +454,8 @@ def run_cuda(args):
         "steps": K, "warmup": args.warmup, "ms_per_step": ms_total / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": f"{w.name}: X {w.dtype} b={b} n={n}, dY b x m={m}, k={k}, per rank"
-                               + ("" if eps is None else f", eps={eps} (dropped {int(dropped.item())} rows)"),
+                               + ("" if eps is None else f", eps={eps} (dropped {int(dropped.item())} rows)")
+                               + ("" if args.dw_dtype == "f32" and args.layout == "nm" else f", dW {args.dw_dtype} {args.layout}"),
                    "l2": "inputs exceed L2 (X %.0f MiB, dY %.0f MiB per step)" % (b * n * e / 2**20, b * m * e / 2**20)
                    if b * n * e > 126 * 2**20 else "inputs fit L2: warm-cache numbers",
                    "parallelism": f"replicas x{world}"},
@@ -445,7 +504,8 @@ def run_layer_loop(args):
     devc = Xs[0].device
     saved = [dict(idx=torch.empty(k, dtype=torch.int32, device=devc), C=torch.empty((k, n), dtype=tdt, device=devc),
                   invn=torch.empty(2 * k, dtype=torch.float32, device=devc),
-                  f=torch.empty(b, dtype=torch.int32, device=devc), alpha=torch.empty(b, dtype=torch.float32, device=devc))
+                  f=torch.empty(b, dtype=torch.int32, device=devc), alpha=torch.empty(b, dtype=torch.float32, device=devc),
+                  sp=pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, dt_code, devc))
              for _ in range(L)]
     dW = torch.empty((n, m), dtype=torch.float32, device=devc)
     ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, dt_code, devc)
@@ -455,10 +515,11 @@ def run_layer_loop(args):
         for l in range(L):
             sv = saved[l]
             pamm.compress_fused(Xs[l % D], k, w.index_seed + 100 * l + s, idx_out=sv["idx"], C=sv["C"], c_invnorm=sv["invn"],
-                                f=sv["f"], alpha=sv["alpha"], stream=stream)
+                                f=sv["f"], alpha=sv["alpha"], sort_products=sv["sp"], stream=stream)
         for l in reversed(range(L)):
             sv = saved[l]
-            pamm.contract_weight_grad(sv["C"], sv["f"], sv["alpha"], dYs[l % D], dW=dW, workspace=ws, stream=stream)
+            pamm.contract_weight_grad(sv["C"], sv["f"], sv["alpha"], dYs[l % D], dW=dW, sort_products=sv["sp"], workspace=ws,
+                                      stream=stream)
 
     for s in range(max(3, args.warmup)):
         step(s)
@@ -478,7 +539,7 @@ def run_layer_loop(args):
     if status != pamm.OK:
         raise SystemExit(f"device status after the timed region: {pamm.status_string(status)}")
     ms = e0.elapsed_time(e1)
-    kept = sum(sum(t.numel() * t.element_size() for key, t in sv.items() if key in ("C", "f", "alpha")) for sv in saved)
+    kept = sum(sum(t.numel() * t.element_size() for key, t in sv.items() if key in ("C", "f", "alpha", "sp")) for sv in saved)
     full = L * b * n * e
     line = {
         "metric": METRIC, "value": b * L * K / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": K,
@@ -508,6 +569,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eps", type=float, default=None,
                     help="time the neighbourhood-condition path (Eq. 2, beta) with this epsilon instead of epsilon = infinity")
+    ap.add_argument("--dw-dtype", choices=["f32", "bf16"], default="f32", help="storage type of the weight gradient")
+    ap.add_argument("--layout", choices=["nm", "mn"], default="nm", help="dW as n x m (the paper's) or m x n (out x in)")
     ap.add_argument("--layers", type=int, default=1,
                     help="with L > 1: a stack of L layers (forward of all, then backward in reverse) and its saved-activation bytes")
     ap.add_argument("--distinct-layers", type=int, default=4, help="distinct synthetic input sets in the --layers mode")

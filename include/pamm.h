@@ -27,8 +27,10 @@
  *    combinations return PAMM_ERR_UNSUPPORTED; there is no CPU fallback.
  *  - Problems only the device can see (a generator index out of range, a
  *    duplicated index, an assignment f_i outside [0,k), a bounded wait that ran
- *    out) never trap: the kernel skips the access, ORs a bit into a per-device
- *    status word and finishes.  Read it with pamm_last_device_status.
+ *    out) never trap: the kernel skips the access, ORs a bit into a status
+ *    word and finishes.  There is ONE word per device, shared by every stream
+ *    (two streams cannot tell their errors apart); read it with
+ *    pamm_last_device_status after synchronising the work you ask about.
  *  - Outputs are fully overwritten.  Results are deterministic: the same
  *    inputs give bit-identical outputs from run to run.
  */
@@ -54,15 +56,29 @@ typedef enum {
 
 typedef enum { PAMM_F32 = 0, PAMM_BF16 = 1 } pamm_dtype;
 
+/* Layout of the weight gradient.  The paper writes O~ = C^T B~ as n x m (hidden
+ * x outputs, Section 3.1); a framework's linear layer usually keeps its weight
+ * as out x in, i.e. m x n. */
+typedef enum { PAMM_DW_NM = 0, PAMM_DW_MN = 1 } pamm_layout;
+
+/* Storage type of the assignment f (Appendix "Complexity Analysis" counts b
+ * scalars for it; with k <= 256 or k <= 65536 generators a byte or two suffice).
+ * Values are 0-based generator indices, unsigned for the narrow types. */
+typedef enum { PAMM_IDX_I32 = 0, PAMM_IDX_U16 = 1, PAMM_IDX_U8 = 2 } pamm_index_type;
+
 /* Which scratch size is asked for. */
 typedef enum {
-    PAMM_WS_COMPRESS = 0,
+    PAMM_WS_COMPRESS = 0,            /* sort products pamm_compress_fused leaves for the backward pass */
     PAMM_WS_CONTRACT = 1,            /* also covers pamm_contract_weight_grad */
     PAMM_WS_STEP_HOST = 2            /* device arena of pamm_qkv_step_host    */
 } pamm_ws_kind;
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* pamm_status_string(pamm_status s);
+
+/* Which CUDA call was behind the calling thread's last PAMM_ERR_CUDA, and the runtime's
+ * name for the failure ("" if there was none).  The string belongs to the library. */
+const char* pamm_last_error_detail(void);
 
 /* Bytes of 256-byte-aligned device scratch the named call needs for these
  * sizes (0 is a valid answer).  Returns (size_t)-1 for invalid sizes. */
@@ -106,12 +122,19 @@ pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_
  *   |csim(X_i, C_j)|, Lemma 1);  alpha_i = S_{i,f_i} / ||C_{f_i}||^2  (Eq. 1).
  * Products are exact, sums are accumulated in fp32.  A zero row gets f = 0,
  * alpha = 0.
- *   f      b int32 (0-based)      alpha  b fp32
- *   workspace  pamm_workspace_bytes(PAMM_WS_COMPRESS, ...) bytes
+ *   f      b entries of f_type, 0-based (k must fit the type: PAMM_ERR_INVALID_ARG otherwise)
+ *   alpha  b fp32
+ *   workspace  NULL, or pamm_workspace_bytes(PAMM_WS_COMPRESS, ...) bytes that receive
+ *          the "sort products": how many rows of every block of rows chose each
+ *          generator, counted on the fly by the pass.  They are an optional by-product
+ *          for the backward pass (pamm_contract, pamm_contract_weight_grad), which then
+ *          skips its own counting launch; they must be kept next to f until then and
+ *          are valid only for this f on a device with the same number of SMs.
  */
 pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
                           const void* C, int64_t ldc, int64_t k, const float* c_invnorm,
-                          int32_t* f, float* alpha, void* workspace, size_t ws_bytes, void* stream);
+                          void* f, pamm_index_type f_type, float* alpha,
+                          void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * Steps 1+2 in one call (Algorithm 2: the Compress call on the flattened X):
@@ -120,7 +143,28 @@ pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm
 pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
                                 int64_t k, uint64_t seed, const int32_t* idx_in,
                                 int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
-                                int32_t* f, float* alpha, void* workspace, size_t ws_bytes, void* stream);
+                                void* f, pamm_index_type f_type, float* alpha,
+                                void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Step 2 for several generator sets at once -- one compression per projection
+ * (Section 4: the method "is applied to the Q, K and V projections"; the worked
+ * example of the appendix "Complexity Analysis" has m = n per projection) -- in ONE
+ * pass over X.  Set s has its k generators in rows [s k, (s+1) k) of C, its norms in
+ * c_invnorm[2 k s, 2 k (s+1)) (fill both with one pamm_select_generators call per
+ * set, each with its own seed), and receives f and alpha at entry offset
+ * s * out_stride.  Every set's result equals what pamm_compress gives for that set
+ * alone.  The backward pass then runs per projection on its own columns of dY and dW
+ * (pamm_contract / pamm_weight_grad with pointer offsets and the leading dimensions).
+ *   sets        1..64
+ *   out_stride  >= b, in entries; out_stride * sizeof(f entry) a multiple of 4
+ *   workspace   NULL or sets * pamm_workspace_bytes(PAMM_WS_COMPRESS, ...) bytes:
+ *               the sort products of set s start at byte s * that size
+ */
+pamm_status pamm_compress_projections(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
+                                      const void* C, int64_t ldc, int64_t k, int64_t sets,
+                                      const float* c_invnorm, void* f, pamm_index_type f_type, float* alpha,
+                                      int64_t out_stride, void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * Step 3 -- contract (Section 3.2 "Approximate Matrix Multiplication";
@@ -132,20 +176,28 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
  * atomics, so the result is reproducible bit for bit.  A row whose f_i is
  * outside [0,k) is skipped and raises PAMM_ERR_BAD_INDEX in the status word.
  *   dY  b x m, dtype dt, leading dimension ldy     Btilde  k x m fp32, ldb
+ *   sort_products  NULL, or what a compress call left in its workspace for this
+ *       very f (same b, k, device).  Counts that belong to another f give a wrong
+ *       B~ and PAMM_ERR_BAD_INDEX in the status word, never an access out of bounds.
  */
-pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy,
-                          int64_t b, int64_t m, pamm_dtype dt, int64_t k,
-                          float* Btilde, int64_t ldb, void* workspace, size_t ws_bytes, void* stream);
+pamm_status pamm_contract(const void* f, pamm_index_type f_type, const float* alpha,
+                          const void* dY, int64_t ldy, int64_t b, int64_t m, pamm_dtype dt, int64_t k,
+                          float* Btilde, int64_t ldb, const void* sort_products,
+                          void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * Step 4 -- weight gradient (Algorithm 1, ApproxMM: the final product; Algorithm 3,
  * the weight gradient through ApproxMM):
- *   dW[r,c] = sum_j C[j,r] * B~[j,c]                          (n x m, fp32)
- *   C  k x n, dtype dt, ldc      Btilde  k x m fp32, ldb      dW  n x m fp32, ldw
+ *   dW[r,c] = sum_j C[j,r] * B~[j,c]
+ *   C  k x n, dtype dt, ldc      Btilde  k x m fp32, ldb
+ *   dW      layout PAMM_DW_NM: n x m (the paper's O~);  PAMM_DW_MN: its transpose,
+ *           m x n (out x in);  leading dimension ldw in elements of dw_dt
+ *   dw_dt   PAMM_F32, or PAMM_BF16 (the fp32 accumulator is rounded to nearest even
+ *           once, on the way out)
  */
 pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
                              const float* Btilde, int64_t ldb, int64_t m,
-                             float* dW, int64_t ldw, void* stream);
+                             void* dW, int64_t ldw, pamm_dtype dw_dt, pamm_layout layout, void* stream);
 
 /*
  * Step 2 with the neighbourhood condition (Section 3.2, Eq. 2; Algorithm 1,
@@ -164,7 +216,7 @@ pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, p
  */
 pamm_status pamm_compress_eps(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
                               const void* C, int64_t ldc, int64_t k, const float* c_invnorm, float eps,
-                              int32_t* f, float* alpha, int32_t* dropped,
+                              void* f, pamm_index_type f_type, float* alpha, int32_t* dropped,
                               void* workspace, size_t ws_bytes, void* stream);
 
 /*
@@ -177,34 +229,37 @@ pamm_status pamm_compress_eps(const void* X, int64_t ldx, int64_t b, int64_t n, 
 pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
                                   const float* Btilde, int64_t ldb, int64_t m,
                                   int64_t b, const int32_t* dropped,
-                                  float* dW, int64_t ldw, void* stream);
+                                  void* dW, int64_t ldw, pamm_dtype dw_dt, pamm_layout layout, void* stream);
 
 /*
  * Step 4, accumulating: dW += C^T B~ (Algorithm 3's weight gradient added to what dW
  * already holds, as gradient accumulation over micro-batches needs).  Every element
  * of dW receives exactly one addition per call, so the result is reproducible.
+ * dW is fp32 (the type gradients are accumulated in), in either layout.
  */
 pamm_status pamm_weight_grad_accumulate(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
                                         const float* Btilde, int64_t ldb, int64_t m,
-                                        float* dW, int64_t ldw, void* stream);
+                                        float* dW, int64_t ldw, pamm_layout layout, void* stream);
 
 /*
  * Steps 3+4 in one call (Algorithm 3, backward of the linear layer, the
  * weight-gradient half): contract dY into B~ and multiply by C^T.  Btilde may
- * be NULL, in which case B~ lives in the workspace only.
+ * be NULL, in which case B~ lives in the workspace only.  dW, dw_dt, layout as in
+ * pamm_weight_grad; sort_products as in pamm_contract.
  */
 pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n,
-                                      const int32_t* f, const float* alpha,
+                                      const void* f, pamm_index_type f_type, const float* alpha,
                                       const void* dY, int64_t ldy, int64_t b, int64_t m, pamm_dtype dt,
                                       int64_t k, float* Btilde, int64_t ldb,
-                                      float* dW, int64_t ldw,
+                                      void* dW, int64_t ldw, pamm_dtype dw_dt, pamm_layout layout,
+                                      const void* sort_products,
                                       void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * The whole path from HOST buffers (Algorithm 2's Compress followed by
  * Algorithm 3's ApproxMM for one layer): copies X and dY host->device into the
- * caller's device arena, runs steps 1-4 there, and copies dW (and, if the
- * pointers are non-NULL, f and alpha) back to the host.  X_host / dY_host /
+ * caller's device arena, runs steps 1-4 there, and copies dW (fp32, n x m; and, if the
+ * pointers are non-NULL, f as int32 and alpha) back to the host.  X_host / dY_host /
  * dW_host should be pinned for the copies to be asynchronous.  `arena` is
  * pamm_workspace_bytes(PAMM_WS_STEP_HOST, ...) bytes of device memory.
  * The call enqueues everything on `stream` and returns; synchronise the stream
@@ -215,6 +270,15 @@ pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host,
                                int64_t k, uint64_t seed,
                                float* dW_host, int32_t* f_host, float* alpha_host,
                                void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * What is kept for the backward pass (appendix "Complexity Analysis": k n + 2 b scalars
+ * instead of b n).  No GPU is touched.
+ *   out[0]  bytes of X (b n elements of dt)
+ *   out[1]  bytes of (C in dt, f in f_type, alpha fp32)
+ *   out[2]  b n, out[3]  k n + 2 b: the paper's scalar counts
+ */
+pamm_status pamm_saved_bytes(int64_t b, int64_t n, int64_t k, pamm_dtype dt, pamm_index_type f_type, int64_t out[4]);
 
 /*
  * Contract without any caller-provided or library-allocated scratch (the paper
@@ -254,9 +318,13 @@ pamm_status pamm_contract_no_alloc(const int32_t* f, const float* alpha, const v
                                    float* Btilde, int64_t ldb, void* stream);
 
 /*
- * Synchronises `stream`, then reads and clears the current device's status
- * word.  Returns PAMM_OK, PAMM_ERR_TIMEOUT, PAMM_ERR_BAD_INDEX, or
- * PAMM_ERR_CUDA if the stream itself reports an error.
+ * Reads and clears the current device's status word WITHOUT waiting for any of the
+ * caller's streams: it reports what kernels that have already finished left there, so
+ * synchronise the work you ask about first.  The word is per device, not per stream;
+ * `stream` is accepted for symmetry with the other calls and not used.  The first
+ * call on a device creates a small private stream and a pinned host word (no device
+ * memory).  Returns PAMM_OK, PAMM_ERR_TIMEOUT, PAMM_ERR_BAD_INDEX, or PAMM_ERR_CUDA
+ * if the read itself failed.
  */
 pamm_status pamm_last_device_status(void* stream);
 

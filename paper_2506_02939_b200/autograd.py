@@ -31,19 +31,27 @@ class PammLinearFunction(torch.autograd.Function):
         n, m = W.shape
         Z = X @ W
         X2 = _rows(X.detach(), n)
-        _, C, _, f, alpha = pamm.compress_fused(X2, int(k), int(seed))
-        ctx.save_for_backward(C, f, alpha, W)          # k n + 2 b scalars instead of b n
+        b = X2.shape[0]
+        f_dtype = torch.uint8 if k <= 256 else torch.int16 if k <= 65536 else torch.int32
+        # the pass also leaves its per-block counts of f (a few KiB): the backward's counting sort starts from them
+        sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, int(k), pamm.BF16 if X2.dtype == torch.bfloat16 else pamm.F32,
+                                  X2.device)
+        _, C, _, f, alpha = pamm.compress_fused(X2, int(k), int(seed), sort_products=sp, f_dtype=f_dtype)
+        ctx.save_for_backward(C, f, alpha, sp, W)      # k n + 2 b scalars instead of b n
         return Z
 
     @staticmethod
     def backward(ctx, dZ):
-        C, f, alpha, W = ctx.saved_tensors
+        C, f, alpha, sp, W = ctx.saved_tensors
         n, m = W.shape
         dX = dZ @ W.t() if ctx.needs_input_grad[0] else None
         dW = None
         if ctx.needs_input_grad[1]:
             dZ2 = _rows(dZ.to(C.dtype), m)
-            dW = pamm.contract_weight_grad(C, f, alpha, dZ2).to(W.dtype)
+            direct = W.dtype in (torch.float32, torch.bfloat16)      # the product kernel writes these itself
+            dW = pamm.contract_weight_grad(C, f, alpha, dZ2, dw_dtype=W.dtype if direct else torch.float32, sort_products=sp)
+            if not direct:
+                dW = dW.to(W.dtype)
         return dX, dW, None, None
 
 

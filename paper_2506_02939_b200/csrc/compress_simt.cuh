@@ -20,7 +20,7 @@ __global__ void __launch_bounds__(CS_THREADS)
 compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
                      const T* __restrict__ C, int64_t ldc, int k,
                      const float* __restrict__ c_invnorm,
-                     int32_t* __restrict__ f, float* __restrict__ alpha, float eps2, float slack,
+                     void* __restrict__ f, int f_type, float* __restrict__ alpha, float eps2, float slack,
                      int32_t* __restrict__ dropped) {
     constexpr int V = Vec16<T>::N;
     const int lane = threadIdx.x & 31;
@@ -81,7 +81,7 @@ compress_simt_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n,
                 a = 0.f;
                 atomicAdd(dropped, 1);
             }
-            f[i] = j_best;
+            store_index(f, f_type, i, j_best);
             alpha[i] = a;
         }
     }

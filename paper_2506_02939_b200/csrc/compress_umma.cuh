@@ -3,8 +3,8 @@
 //
 // One streaming pass over X.  The rows are cut into equal contiguous ranges, one
 // per CTA (one CTA per SM, a single balanced wave).  Inside a CTA:
-//   warp 0     TMA producer: X tiles (32-row boxes, so a ragged last tile costs
-//              only the bytes it needs) and the matching C tile, 64 columns of
+//   warp 0     TMA producer: X tiles (64-row boxes, so a ragged last tile costs
+//              only the boxes it needs) and the matching C tile, 64 columns of
 //              the hidden dimension per pipeline stage, 128-byte swizzle
 //   warp 1     issues tcgen05.mma (M = 128 rows, N = generators of the chunk,
 //              K = 16 per instruction), fp32 accumulators in TMEM, two buffers
@@ -21,7 +21,16 @@
 //              ||X_i||^2 - S^2/||C_f||^2 > eps^2 ||X_i||^2 (+ a rounding allowance)
 // C is small (k x n) and is re-read per row tile from L2; with MT = 2 two row
 // tiles share every C tile.  For k > 256 the generators are processed in chunks
-// with a running (best score, argmax, dot product) per row.
+// with a running (best score, argmax, dot product) per row; X is then fetched once
+// per chunk, from HBM the first time and from L2 afterwards (only the last pass
+// over a tile carries the evict-first hint).
+//
+// Several independent generator sets ("groups": one compression per projection,
+// Section 4) are served by the same pass: the chunks of all groups follow one
+// another, the running argmax restarts at every group, and every group gets its
+// own f and alpha.  The epilogue also counts, per CTA and group, how many rows
+// chose each generator (integer atomics in shared memory): the per-block histograms
+// the backward pass's counting sort starts from.
 #pragma once
 #include "pamm_common.cuh"
 #include "sm100_ptx.cuh"
@@ -32,19 +41,17 @@ __host__ __device__ constexpr int CU_THREADS(int mt) { return 64 + mt * 128; }  
 __host__ __device__ constexpr int CU_THREADS_EPS(int mt) { return 64 + mt * 256; }     // + one thread per row for ||X_i||^2
 constexpr int CU_BLOCK_K = 64;                 // bf16 columns per stage = one 128-byte swizzle row
 constexpr int CU_TILE_M = 128;
-#ifndef PAMM_CU_BOX_ROWS
-#define PAMM_CU_BOX_ROWS 64
-#endif
-constexpr int CU_BOX_ROWS = PAMM_CU_BOX_ROWS;
+constexpr int CU_BOX_ROWS = 64;                // rows per TMA box of X (a ragged last tile fetches only the boxes it needs)
 constexpr int CU_X_TILE_BYTES = CU_TILE_M * 128;   // 16 KiB
 constexpr int CU_MAX_K = 4096;                 // 1/||C_j|| and 1/||C_j||^2 live in shared memory
-constexpr int CU_SMEM_BUDGET = 200 * 1024;
+constexpr int CU_SMEM_BUDGET = 200 * 1024;     // pipeline stages: more than this buys nothing
+constexpr size_t CU_SMEM_LIMIT = 227 * 1024;   // dynamic + static shared memory a CTA may have
 
 struct CompressUmmaPlan {
-    int mt;            // row tiles (of 128) per super tile: 2 when the chunk has <= 128 generators
+    int mt;            // row tiles (of 128) per super tile
     int n_chunk;       // generators per chunk, padded to a multiple of 16 (<= 256)
-    int num_chunks;
-    int stages;
+    int num_chunks;    // chunks per group
+    int stages;        // 0 when the shared memory does not allow two stages
     int stage_bytes;
     int tmem_cols;
     int tmem_bufs;
@@ -57,26 +64,33 @@ inline bool compress_umma_supported(int64_t b, int64_t n, int64_t k) {
     return k >= 16 && k <= CU_MAX_K && n >= 8 && b >= 1 && n < (1ll << 31);
 }
 
-inline CompressUmmaPlan compress_umma_plan(int64_t b, int64_t k, int sms) {
+// Rows per CTA of the streaming pass: equal contiguous ranges, a multiple of the TMA box.
+// The same partition is used for the per-block histograms of f.
+inline int compress_rows_per_cta(int64_t b, int sms) {
+    const int64_t per = (b + sms - 1) / sms;
+    return (int)std::min<int64_t>(std::max<int64_t>(CU_BOX_ROWS, round_up(per, CU_BOX_ROWS)), 1ll << 30);
+}
+
+// static_smem: the kernel's statically declared shared memory (barriers, row norms).
+inline CompressUmmaPlan compress_umma_plan(int64_t b, int64_t k, int groups, int sms, size_t static_smem) {
     CompressUmmaPlan p;
     const int npad = (int)round_up(k, 16);
     p.num_chunks = (npad + 255) / 256;
     p.n_chunk = (int)round_up((npad + p.num_chunks - 1) / p.num_chunks, 16);
-#ifdef PAMM_CU_MT1_WIDE
-    p.mt = p.n_chunk <= 128 ? 2 : 1;
-#else
     p.mt = 2;      // two row tiles share every C tile; beyond 128 generators per chunk they fill TMEM (one buffer)
-#endif
     p.stage_bytes = p.mt * CU_X_TILE_BYTES + p.n_chunk * 128;
-    p.stages = std::min(8, CU_SMEM_BUDGET / p.stage_bytes);
+    // 1/||C||, 1/||C||^2 and the histogram of every group, the 1024-byte alignment slack
+    const size_t fixed = 1024 + (size_t)groups * (p.num_chunks * p.n_chunk + 2 * k) * 4 + 256;
+    const size_t budget = CU_SMEM_LIMIT > fixed + static_smem ? CU_SMEM_LIMIT - fixed - static_smem : 0;
+    p.stages = (int)std::min<size_t>(8, std::min<size_t>(CU_SMEM_BUDGET, budget) / p.stage_bytes);
+    if (p.stages < 2) p.stages = 0;
     p.tmem_bufs = 2 * p.mt * p.n_chunk <= 512 ? 2 : 1;     // accumulator sets: the epilogue overlaps the next MMAs only with two
     int cols = p.tmem_bufs * p.mt * p.n_chunk;
     p.tmem_cols = 32;
     while (p.tmem_cols < cols) p.tmem_cols *= 2;
-    const int64_t per = (b + sms - 1) / sms;
-    p.rows_per_cta = (int)std::max<int64_t>(CU_BOX_ROWS, round_up(per, CU_BOX_ROWS));
+    p.rows_per_cta = compress_rows_per_cta(b, sms);
     p.grid = (int)((b + p.rows_per_cta - 1) / p.rows_per_cta);
-    p.smem_bytes = 1024 + (size_t)p.stages * p.stage_bytes + (size_t)(p.num_chunks * p.n_chunk + k) * 4 + 256;
+    p.smem_bytes = fixed + (size_t)p.stages * p.stage_bytes;
     return p;
 }
 
@@ -117,33 +131,46 @@ __device__ __forceinline__ void argmax16(const uint32_t (&v)[16], const float* _
 // its generator's line (distance 0) is kept for every eps >= 0.
 __host__ __device__ inline float neighbourhood_slack(int64_t n) { return 2.f * (float)n * 5.9604645e-8f; }
 
+// What the compress kernel writes besides alpha.
+struct CompressOut {
+    void* f;                 // groups x out_stride entries of `f_type` (a pamm_index_type)
+    float* alpha;            // groups x out_stride
+    int64_t out_stride;      // distance between two groups' vectors, in entries
+    int32_t* hist;           // per group, gridDim.x x k counts of f per CTA; or nullptr
+    int64_t hist_stride;     // distance between two groups' tables, in counts
+    int f_type;
+};
+
 // EPS = false: the paper's setting (epsilon = infinity), nothing is dropped.
-// EPS = true : eps2 = epsilon^2 and slack as above; *dropped counts the dropped rows.
+// EPS = true : eps2 = epsilon^2 and slack as above; *dropped counts the dropped rows (one group only).
+// C holds the generators of all groups, group g in rows [g k, (g+1) k); c_invnorm holds 2k
+// entries per group (1/||C_j||, then 1/||C_j||^2).
 template <int MT, bool EPS>
 __global__ void __launch_bounds__(EPS ? CU_THREADS_EPS(MT) : CU_THREADS(MT), 1)
 compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_c,
-                     int64_t b, int n, int k, int n_chunk, int num_chunks, int stages, int stage_bytes,
+                     int64_t b, int n, int k, int groups, int n_chunk, int num_chunks, int stages, int stage_bytes,
                      int tmem_cols, int tmem_bufs, int rows_per_cta, int x_is_ready, const float* __restrict__ c_invnorm,
-                     int32_t* __restrict__ f, float* __restrict__ alpha, float eps2, float slack,
-                     int32_t* __restrict__ dropped) {
+                     CompressOut out, float eps2, float slack, int32_t* __restrict__ dropped) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2], s_nfull[2], s_nempty[2];
-    __shared__ float s_norm[2][MT * CU_TILE_M];     // ||X_i||^2 of the rows of a super tile (EPS only)
+    __shared__ float s_norm[EPS ? 2 : 1][EPS ? MT * CU_TILE_M : 1];     // ||X_i||^2 of the rows of a super tile (EPS only)
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    // 1/||C_j|| for every column the chunks cover, zero beyond k (a padded column scores 0
-    // and never beats a real one), then 1/||C_j||^2
+    // per group: 1/||C_j|| for every column the chunks cover, zero beyond k (a padded column
+    // scores 0 and never beats a real one); then 1/||C_j||^2; then the histogram of f
     const int kpad = n_chunk * num_chunks;
     float* s_inv = reinterpret_cast<float*>(tiles + (size_t)stages * stage_bytes);
-    float* s_inv2 = s_inv + kpad;
+    float* s_inv2 = s_inv + groups * kpad;
+    int32_t* s_hist = reinterpret_cast<int32_t*>(s_inv2 + groups * k);
 
     const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
     const int64_t r1 = min(b, r0 + (int64_t)rows_per_cta);
     const int ksteps = (n + CU_BLOCK_K - 1) / CU_BLOCK_K;
     const int super_rows = MT * CU_TILE_M;
+    const int passes = groups * num_chunks;          // passes over a super tile of X: one per (group, chunk)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&s_empty[s], EPS ? 1 + 4 * MT : 1); }
@@ -161,7 +188,11 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         ptx::tmem_alloc(&s_tmem_base, (uint32_t)tmem_cols);
         ptx::tmem_relinquish();
     }
-    grid_launch_dependents();   // the next kernel of the stream may set itself up meanwhile
+    // The next kernel of the stream may set itself up meanwhile.  It is released before this
+    // kernel's own wait: its grid_dependency_wait() still covers everything older (see the
+    // rule beside grid_dependency_wait), and it must not touch f, alpha or the histograms
+    // before that wait.
+    grid_launch_dependents();
     // C and the norms come from the kernel before.  When the caller vouches that X was
     // complete before that kernel started, the producer streams the first X tiles while
     // it still runs and everybody else waits for it only where C or the norms are read.
@@ -178,12 +209,13 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             ptx::prefetch_tensormap(&tm_x);
             ptx::prefetch_tensormap(&tm_c);
             const uint64_t stream_policy = ptx::l2_policy_evict_first();   // X is read once; C stays in L2
-            // pipeline step `it` = (row super tile, generator chunk, 64-column step), flattened
-            const uint32_t per_super = (uint32_t)(num_chunks * ksteps);
+            // pipeline step `it` = (row super tile, pass = (group, chunk), 64-column step), flattened
+            const uint32_t per_super = (uint32_t)(passes * ksteps);
             const uint32_t total = (uint32_t)((r1 - r0 + super_rows - 1) / super_rows) * per_super;
             auto issue = [&](uint32_t at, bool with_x, bool with_c, bool arm) {
                 const int64_t st = r0 + (int64_t)(at / per_super) * super_rows;
-                const int ch = (int)((at % per_super) / (uint32_t)ksteps), ks = (int)(at % (uint32_t)ksteps);
+                const int pass = (int)((at % per_super) / (uint32_t)ksteps), ks = (int)(at % (uint32_t)ksteps);
+                const int g = pass / num_chunks, ch = pass % num_chunks;
                 const int s = at % stages;
                 uint8_t* stage = tiles + (size_t)s * stage_bytes;
                 uint32_t bytes = (uint32_t)n_chunk * 128u;
@@ -196,15 +228,19 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                 }
                 if (arm) ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
                 if (with_x) {
+                    // the tile comes back once per pass: only its last visit may push it out of L2 early
+                    const bool last_pass = pass + 1 == passes;
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
-                        for (int q = 0; q < boxes[mt]; ++q)
-                            ptx::tma_load_2d_hint(stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128), &tm_x,
-                                                  ks * CU_BLOCK_K, (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS),
-                                                  &s_full[s], stream_policy);
+                        for (int q = 0; q < boxes[mt]; ++q) {
+                            uint8_t* dst = stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128);
+                            const int32_t y = (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS);
+                            if (last_pass) ptx::tma_load_2d_hint(dst, &tm_x, ks * CU_BLOCK_K, y, &s_full[s], stream_policy);
+                            else           ptx::tma_load_2d(dst, &tm_x, ks * CU_BLOCK_K, y, &s_full[s]);
+                        }
                 }
                 if (with_c)
-                    ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, ch * n_chunk, &s_full[s]);
+                    ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, g * k + ch * n_chunk, &s_full[s]);
             };
             uint32_t it = 0;
             bool ok = true;
@@ -238,7 +274,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             uint32_t it = 0, unit = 0;
             bool ok = true;
             for (int64_t st = r0; st < r1 && ok; st += super_rows) {
-                for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
+                for (int pass = 0; pass < passes && ok; ++pass, ++unit) {
                     const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
                     if (!ptx::mbar_wait(&s_tempty[buf], uph ^ 1u, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
@@ -269,7 +305,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         // ---------------- squared row norms: one row of the super tile per thread ----------------
         const int nt = threadIdx.x - CU_THREADS(MT);
         const int my_mt = nt / CU_TILE_M, row_in_tile = nt % CU_TILE_M;
-        const int ksteps_all = num_chunks * ksteps;
+        const int ksteps_all = passes * ksteps;
         uint32_t it = 0, sup = 0;
         bool ok = true;
         for (int64_t st = r0; st < r1 && ok; st += super_rows, ++sup) {
@@ -279,7 +315,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                 const int s = it % stages;
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[s], (it / stages) & 1u, abort_flag));   // warp-uniform
                 if (!ok) break;
-                if (q < ksteps && live) {     // the first generator chunk sees every column of X once
+                if (q < ksteps && live) {     // the first pass sees every column of X once
                     const uint8_t* rowp = tiles + (size_t)s * stage_bytes + my_mt * CU_X_TILE_BYTES + row_in_tile * 128;
                     uint4 w[8];
 #pragma unroll
@@ -313,57 +349,64 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
         const int mt = (warp - 2) >> 2;                  // my row tile of the super tile
         const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
+        for (int j = threadIdx.x - 64; j < groups * k; j += 128 * MT) s_hist[j] = 0;
         if (x_is_ready) grid_dependency_wait();
-        for (int j = threadIdx.x - 64; j < kpad; j += 128 * MT) s_inv[j] = j < k ? c_invnorm[j] : 0.f;
-        for (int j = threadIdx.x - 64; j < k; j += 128 * MT) s_inv2[j] = c_invnorm[k + j];
+        for (int j = threadIdx.x - 64; j < groups * kpad; j += 128 * MT) {
+            const int g = j / kpad, jj = j % kpad;
+            s_inv[j] = jj < k ? c_invnorm[(size_t)g * 2 * k + jj] : 0.f;
+        }
+        for (int j = threadIdx.x - 64; j < groups * k; j += 128 * MT) s_inv2[j] = c_invnorm[(size_t)(j / k) * 2 * k + k + j % k];
         ptx::named_barrier(1, 128 * MT);                 // the epilogue warps share the norms
         uint32_t unit = 0, sup = 0;
         bool ok = true;
         for (int64_t st = r0; st < r1 && ok; st += super_rows, ++sup) {
-            float best = -1.f, s_best = 0.f;
-            int j_best = 0;
             const bool live = st + (int64_t)mt * CU_TILE_M < r1;
-            for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
-                const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_tfull[buf], uph, abort_flag));   // warp-uniform
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                if (live) {
-                    // two register buffers: the TMEM load of the next 16 columns is in flight
-                    // while the current 16 go through the tournament
-                    const uint32_t t_base = tmem_base + buf * (uint32_t)(MT * n_chunk) + lane_base + (uint32_t)(mt * n_chunk);
-                    const int jb = ch * n_chunk;
-                    uint32_t va[16], vb[16];
-                    ptx::tmem_ld_16cols(t_base, va);
-                    for (int c0 = 0; c0 < n_chunk; c0 += 32) {
-                        ptx::tmem_ld_wait(va);
-                        const bool second = c0 + 16 < n_chunk;
-                        if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
-                        argmax16(va, s_inv + jb + c0, jb + c0, best, s_best, j_best);
-                        if (second) {
-                            ptx::tmem_ld_wait(vb);
-                            if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
-                            argmax16(vb, s_inv + jb + c0 + 16, jb + c0 + 16, best, s_best, j_best);
+            const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
+            for (int g = 0; g < groups && ok; ++g) {
+                float best = -1.f, s_best = 0.f;
+                int j_best = 0;
+                for (int ch = 0; ch < num_chunks && ok; ++ch, ++unit) {
+                    const uint32_t buf = unit % (uint32_t)tmem_bufs, uph = (unit / (uint32_t)tmem_bufs) & 1u;
+                    ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_tfull[buf], uph, abort_flag));   // warp-uniform
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    if (live) {
+                        // two register buffers: the TMEM load of the next 16 columns is in flight
+                        // while the current 16 go through the tournament
+                        const uint32_t t_base = tmem_base + buf * (uint32_t)(MT * n_chunk) + lane_base + (uint32_t)(mt * n_chunk);
+                        const int jb = ch * n_chunk;
+                        const float* inv = s_inv + g * kpad + jb;
+                        uint32_t va[16], vb[16];
+                        ptx::tmem_ld_16cols(t_base, va);
+                        for (int c0 = 0; c0 < n_chunk; c0 += 32) {
+                            ptx::tmem_ld_wait(va);
+                            const bool second = c0 + 16 < n_chunk;
+                            if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
+                            argmax16(va, inv + c0, jb + c0, best, s_best, j_best);
+                            if (second) {
+                                ptx::tmem_ld_wait(vb);
+                                if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
+                                argmax16(vb, inv + c0 + 16, jb + c0 + 16, best, s_best, j_best);
+                            }
                         }
                     }
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
                 }
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
-            }
-            if (ok && EPS) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_nfull[sup & 1u], (sup >> 1) & 1u, abort_flag));
-            if (ok) {
+                if (ok && EPS) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_nfull[sup & 1u], (sup >> 1) & 1u, abort_flag));
+                if (!ok) break;
                 int ndrop = 0;
-                const int64_t row = st + (int64_t)mt * CU_TILE_M + quad * 32 + lane;
                 if (row < r1) {
-                    float a = s_best * s_inv2[j_best];
+                    float a = s_best * s_inv2[g * k + j_best];
                     if (EPS) {     // Eq. 2: ||X_i - alpha C_f||^2 = ||X_i||^2 - S^2/||C_f||^2 against eps^2 ||X_i||^2
                         const float nx = s_norm[sup & 1u][mt * CU_TILE_M + quad * 32 + lane];
                         const float dist2 = nx - s_best * a;
                         if (dist2 > (eps2 + slack) * nx) { a = 0.f; ++ndrop; }
                     }
-                    f[row] = j_best;
-                    alpha[row] = a;
+                    store_index(out.f, out.f_type, (int64_t)g * out.out_stride + row, j_best);
+                    out.alpha[(int64_t)g * out.out_stride + row] = a;
+                    atomicAdd(&s_hist[g * k + j_best], 1);
                 }
                 if (EPS) {
                     __syncwarp();
@@ -375,6 +418,14 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             }
         }
         if (!ok && lane == 0) raise_status(DEV_TIMEOUT);
+        // this CTA's histograms of f, one row of the per-block table per group
+        ptx::named_barrier(1, 128 * MT);
+        if (out.hist) {
+            for (int j = threadIdx.x - 64; j < groups * k; j += 128 * MT) {
+                const int g = j / k, jj = j % k;
+                out.hist[(int64_t)g * out.hist_stride + (int64_t)blockIdx.x * k + jj] = s_hist[j];
+            }
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -385,17 +436,38 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     }
 }
 
+template <int MT, bool EPS>
+inline size_t compress_umma_static_smem() {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, compress_umma_kernel<MT, EPS>) != cudaSuccess) return 4096;
+    return fa.sharedSizeBytes;
+}
+
+// The plan for these sizes, with the kernel's own static shared memory taken into account.
+inline CompressUmmaPlan compress_umma_plan_for(int64_t b, int64_t k, int groups, int sms, bool with_eps) {
+    static size_t st_plain = 0, st_eps = 0;     // the same on every device
+    if (!st_plain) st_plain = compress_umma_static_smem<2, false>();
+    if (!st_eps) st_eps = compress_umma_static_smem<2, true>();
+    return compress_umma_plan(b, k, groups, sms, with_eps ? st_eps : st_plain);
+}
+
+// Whether the tensor-core kernel serves these sizes (else the CUDA-core kernel does).
+inline bool compress_umma_usable(int64_t b, int64_t n, int64_t k, int groups, int sms, bool with_eps) {
+    return compress_umma_supported(b, n, k) && (int64_t)groups * k <= (1 << 20) &&
+           compress_umma_plan_for(b, k, groups, sms, with_eps).stages >= 2;
+}
+
 inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
-                                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, int sms,
+                                        int64_t k, int groups, const float* c_invnorm, const CompressOut& out, int sms,
                                         bool x_is_ready, cudaStream_t st, bool with_eps = false, float eps = 0.f,
                                         int32_t* dropped = nullptr) {
-    const CompressUmmaPlan p = compress_umma_plan(b, k, sms);
+    const CompressUmmaPlan p = compress_umma_plan_for(b, k, groups, sms, with_eps);
+    if (p.stages < 2) return PAMM_ERR_UNSUPPORTED;
     CUtensorMap tm_x, tm_c;
     if (!make_tmap_bf16_sw128(&tm_x, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, CU_BOX_ROWS) ||
-        !make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)p.n_chunk))
-        return PAMM_ERR_CUDA;
-    auto kern = with_eps ? (p.mt == 2 ? compress_umma_kernel<2, true> : compress_umma_kernel<1, true>)
-                         : (p.mt == 2 ? compress_umma_kernel<2, false> : compress_umma_kernel<1, false>);
+        !make_tmap_bf16_sw128(&tm_c, C, (uint64_t)groups * (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)p.n_chunk))
+        return tensor_map_failed();
+    auto kern = with_eps ? compress_umma_kernel<2, true> : compress_umma_kernel<2, false>;
     if (!ensure_dynamic_smem((const void*)kern, p.smem_bytes)) return PAMM_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
@@ -407,10 +479,10 @@ inline pamm_status launch_compress_umma(const void* X, int64_t ldx, int64_t b, i
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
-                       p.tmem_cols, p.tmem_bufs, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, f, alpha, eps * eps,
+    cudaLaunchKernelEx(&cfg, kern, tm_x, tm_c, b, (int)n, (int)k, groups, p.n_chunk, p.num_chunks, p.stages, p.stage_bytes,
+                       p.tmem_cols, p.tmem_bufs, p.rows_per_cta, x_is_ready ? 1 : 0, c_invnorm, out, eps * eps,
                        neighbourhood_slack(n), dropped);
-    return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA;
+    return launch_result("compress_umma_kernel launch");
 }
 
 }  // namespace pamm

@@ -1,7 +1,9 @@
 // Step 3: B~[j,:] = sum_{i: f_i = j} alpha_i * dY[i,:]  (Algorithm 1 ApproxMM,
 // the alpha-scaling of B and the index_add), as a deterministic segmented reduction.
 //
-//   hist    : per block of SORT_BLK rows, a histogram of f            (integers)
+//   hist    : per block of rows, a histogram of f (integers).  The blocks are the row
+//             ranges of the compress pass, whose epilogue already counted f: when the
+//             caller hands those counts over, this launch is skipped
 //   scan    : exclusive scans -> segment starts and per-block offsets
 //   scatter : stable counting sort of row ids by f  -> perm
 //   main    : the sorted rows are cut into equal contiguous ranges, one per CTA
@@ -19,32 +21,28 @@
 
 namespace pamm {
 
-constexpr int SORT_BLK = 1024;         // rows per histogram / scatter block
+constexpr int SORT_BLK = 1024;         // threads of a histogram / scatter block: it walks its rows 1024 at a time
 constexpr int CT_TILE = 256;           // rows of (perm, alpha) staged in shared memory at a time
 constexpr int64_t CT_MAX_K = 49152;    // k * 4 bytes of dynamic shared memory in hist / scatter
-#ifndef PAMM_CT_UNROLL
-#define PAMM_CT_UNROLL 8
-#endif
-#ifndef PAMM_CT_MAX_THREADS
-#define PAMM_CT_MAX_THREADS 768
-#endif
-constexpr int CT_MAX_THREADS = PAMM_CT_MAX_THREADS;
-constexpr int CT_UNROLL = PAMM_CT_UNROLL;     // rows in flight per thread
+constexpr int CT_MAX_THREADS = 768;
+constexpr int CT_UNROLL = 8;           // rows in flight per thread
 constexpr int CT_MAX_CTAS = 148 * 8;   // upper bound on row ranges (sizes the partial buffer)
 
 struct ContractWs {
-    int32_t* hist;        // NB x k   (counts, then exclusive per-block offsets)
+    int32_t* hist;        // NB x k   (counts; the three-launch sort turns them into exclusive per-block offsets)
     int32_t* seg_start;   // k + 1
     int32_t* perm;        // b
     float* partials;      // (CT_MAX_CTAS + k) x m_pad
     float* btilde;        // k x m_pad (used when the caller passes no B~)
-    int64_t nb, m_pad;
+    int64_t nb, rows_per_block, m_pad;
     size_t bytes;
 };
 
-inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k) {
+// rows_per_block: the row partition of the histograms (compress_rows_per_cta).
+inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k, int64_t rows_per_block) {
     ContractWs w;
-    w.nb = (b + SORT_BLK - 1) / SORT_BLK;
+    w.rows_per_block = rows_per_block;
+    w.nb = (b + rows_per_block - 1) / rows_per_block;
     w.m_pad = round_up(m, 4);
     char* p = (char*)base;
     size_t off = 0;
@@ -59,15 +57,17 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
 }
 
 __global__ void __launch_bounds__(SORT_BLK)
-contract_hist_kernel(const int32_t* __restrict__ f, int64_t b, int k, int32_t* __restrict__ hist) {
+contract_hist_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
+                     int32_t* __restrict__ hist) {
     extern __shared__ int32_t s_hist[];
     for (int j = threadIdx.x; j < k; j += SORT_BLK) s_hist[j] = 0;
     grid_dependency_wait();     // f may come from the kernel before
     grid_launch_dependents();
     __syncthreads();
-    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + threadIdx.x;
-    if (i < b) {
-        const int32_t j = f[i];
+    const int64_t i0 = (int64_t)blockIdx.x * rows_per_block;
+    const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
+    for (int64_t i = i0 + threadIdx.x; i < i1; i += SORT_BLK) {
+        const int32_t j = load_index(f, f_type, i);
         if (j >= 0 && j < k) atomicAdd(&s_hist[j], 1);
         else raise_status(DEV_BAD_INDEX);
     }
@@ -128,39 +128,58 @@ contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restr
     if (tid == 0) seg_start[k] = s_carry;
 }
 
-// Stable scatter: rows of one block are ranked warp by warp (ascending row
-// order); inside a warp, match_any groups equal keys and the lowest lane of a
-// group reserves the group's slots.
+// Stable ranking of up to SORT_BLK rows of one block, warp by warp in ascending row
+// order: inside a warp, match_any groups equal keys and the lowest lane of a group
+// reserves the group's slots in s_next.  A slot outside [0, b) can only come from counts
+// that do not belong to this f (a caller's mistake): it is skipped and reported.
+__device__ __forceinline__ void scatter_chunk(int32_t key, int64_t i, int nrows, int32_t* s_next,
+                                              int32_t* __restrict__ perm, int64_t b) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned peers = __match_any_sync(0xffffffffu, key);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    const int leader = __ffs(peers) - 1;
+    const int count = __popc(peers);
+    const int warps = (nrows + 31) >> 5;
+    for (int w = 0; w < warps; ++w) {
+        __syncthreads();
+        if (warp == w) {
+            int32_t base = 0;
+            if (lane == leader && key >= 0) {
+                base = s_next[key];
+                s_next[key] = base + count;
+            }
+            base = __shfl_sync(0xffffffffu, base, leader);
+            if (key >= 0) {
+                const int64_t pos = (int64_t)base + rank;
+                if (pos >= 0 && pos < b) perm[pos] = (int32_t)i;
+                else raise_status(DEV_BAD_INDEX);
+            }
+        }
+    }
+    __syncthreads();
+}
+
+// Stable scatter of one block's rows, given the scanned tables.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const int32_t* __restrict__ hist,
-                        const int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
+contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
+                        const int32_t* __restrict__ hist, const int32_t* __restrict__ seg_start,
+                        int32_t* __restrict__ perm) {
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int32_t* my_hist = hist + (int64_t)blockIdx.x * k;
     grid_dependency_wait();
     grid_launch_dependents();
     for (int j = tid; j < k; j += SORT_BLK) s_next[j] = seg_start[j] + my_hist[j];
-    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
-    int32_t j = -1;
-    if (i < b) {
-        j = f[i];
-        if (j < 0 || j >= k) j = -1;
-    }
-    const unsigned peers = __match_any_sync(0xffffffffu, j);
-    const int rank = __popc(peers & ((1u << lane) - 1u));
-    const int leader = __ffs(peers) - 1;
-    const int count = __popc(peers);
-    for (int w = 0; w < SORT_BLK / 32; ++w) {
-        __syncthreads();
-        if (warp == w) {
-            int32_t base = 0;
-            if (lane == leader && j >= 0) {
-                base = s_next[j];
-                s_next[j] = base + count;
-            }
-            base = __shfl_sync(0xffffffffu, base, leader);
-            if (j >= 0) perm[base + rank] = (int32_t)i;
+    const int64_t i0 = (int64_t)blockIdx.x * rows_per_block;
+    const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
+    for (int64_t c0 = i0; c0 < i1; c0 += SORT_BLK) {
+        const int64_t i = c0 + tid;
+        int32_t key = -1;
+        if (i < i1) {
+            key = load_index(f, f_type, i);
+            if (key < 0 || key >= k) key = -1;
         }
+        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), s_next, perm, b);
     }
 }
 
@@ -174,28 +193,16 @@ contract_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const i
 // threads: with W = the chunk's width rounded up to a power of two, the SORT_BLK
 // / W thread groups each take every (SORT_BLK / W)-th histogram row.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, const int32_t* __restrict__ hist,
-                             int nb, int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
+contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
+                             const int32_t* __restrict__ hist, int nb, int32_t* __restrict__ seg_start,
+                             int32_t* __restrict__ perm) {
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
     __shared__ int32_t s_part[2][SORT_BLK];   // per-thread partial (total, before) of the column sums
     __shared__ int32_t s_warp[32];
     __shared__ int32_t s_carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int me = blockIdx.x;
-    // f is older than the histogram kernel, which did not let this kernel in before its
-    // own wait for f's producer had returned: the keys can be fetched and ranked inside
-    // their warp before this kernel waits for the histograms.
-    const int64_t i = (int64_t)blockIdx.x * SORT_BLK + tid;
-    int32_t key = -1;
-    if (i < b) {
-        key = f[i];
-        if (key < 0 || key >= k) key = -1;
-    }
-    const unsigned peers = __match_any_sync(0xffffffffu, key);
-    const int rank = __popc(peers & ((1u << lane) - 1u));
-    const int leader = __ffs(peers) - 1;
-    const int count = __popc(peers);
-    grid_dependency_wait();
+    grid_dependency_wait();     // f and the histograms come from kernels before
     grid_launch_dependents();
     if (tid == 0) s_carry = 0;
     __syncthreads();
@@ -267,17 +274,16 @@ contract_scan_scatter_kernel(const int32_t* __restrict__ f, int64_t b, int k, co
     }
     if (me == 0 && tid == 0) seg_start[k] = s_carry;
 
-    for (int w = 0; w < SORT_BLK / 32; ++w) {
-        __syncthreads();
-        if (warp == w) {
-            int32_t base = 0;
-            if (lane == leader && key >= 0) {
-                base = s_next[key];
-                s_next[key] = base + count;
-            }
-            base = __shfl_sync(0xffffffffu, base, leader);
-            if (key >= 0) perm[base + rank] = (int32_t)i;
+    const int64_t i0 = (int64_t)me * rows_per_block;
+    const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
+    for (int64_t c0 = i0; c0 < i1; c0 += SORT_BLK) {
+        const int64_t i = c0 + tid;
+        int32_t key = -1;
+        if (i < i1) {
+            key = load_index(f, f_type, i);
+            if (key < 0 || key >= k) key = -1;
         }
+        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), s_next, perm, b);
     }
 }
 
@@ -309,7 +315,7 @@ __device__ __forceinline__ void fma_raw<__nv_bfloat16>(float (&acc)[8], float a,
 
 template <typename T>
 __global__ void __launch_bounds__(CT_MAX_THREADS)
-contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, int64_t ldy, int64_t m,
+contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, int64_t ldy, int64_t b, int64_t m,
                      int k, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ perm,
                      int rows_per_cta, float* __restrict__ partials, int64_t m_pad,
                      float* __restrict__ Bt, int64_t ldb) {
@@ -319,7 +325,7 @@ contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, 
     const int c = blockIdx.x;
     grid_dependency_wait();
     grid_launch_dependents();
-    const int32_t total = seg_start[k];
+    const int32_t total = (int32_t)min((int64_t)max(seg_start[k], 0), b);
     const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
     const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
     if (r_begin >= r_end) return;
@@ -358,9 +364,11 @@ contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, 
         const int tcnt = min(CT_TILE, r_end - t0);
         __syncthreads();
         for (int t = threadIdx.x; t < tcnt; t += blockDim.x) {
-            const int32_t i = perm[t0 + t];
+            int32_t i = perm[t0 + t];
+            const bool bad = (uint32_t)i >= (uint32_t)b;     // only if the sort was fed counts of another f
+            if (bad) { raise_status(DEV_BAD_INDEX); i = 0; }
             s_row[t] = i;
-            s_alpha[t] = alpha[i];
+            s_alpha[t] = bad ? 0.f : alpha[i];
         }
         __syncthreads();
         int pos = 0;
@@ -393,7 +401,7 @@ contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, 
 #pragma unroll
                 for (int e = 0; e < V; ++e) acc[e] = 0.f;
                 if (j_end >= r_end) { j = -1; break; }
-                do { ++j; j_end = seg_start[j + 1]; } while (j_end <= t0 + pos);   // skip empty segments
+                do { ++j; j_end = seg_start[j + 1]; } while (j_end <= t0 + pos && j + 1 < k);   // skip empty segments
             }
         }
         if (j < 0) break;
@@ -406,7 +414,7 @@ constexpr int RED_THREADS = 256;
 // Finishes B~: zero rows for empty segments, sums of partial rows for segments
 // that were cut by a range boundary; rows written directly by main are left alone.
 __global__ void __launch_bounds__(RED_THREADS)
-contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k,
+contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k, int64_t b,
                        const int32_t* __restrict__ seg_start, int rows_per_cta,
                        float* __restrict__ Bt, int64_t ldb) {
     const int64_t mv = m_pad / 4;
@@ -416,7 +424,7 @@ contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_
     if (idx >= (int64_t)k * mv) return;
     const int j = (int)(idx / mv);
     const int64_t col = (idx % mv) * 4;
-    const int32_t s0 = seg_start[j], s1 = seg_start[j + 1];
+    const int32_t s0 = (int32_t)min((int64_t)max(seg_start[j], 0), b), s1 = (int32_t)min((int64_t)max(seg_start[j + 1], 0), b);
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     if (s1 > s0) {
         const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;

@@ -27,30 +27,15 @@
 
 namespace pamm {
 
-#ifndef PAMM_CS_MAX_CONSUMERS
-#define PAMM_CS_MAX_CONSUMERS 384
-#endif
-#ifndef PAMM_CS_RING_KB
-#define PAMM_CS_RING_KB 88
-#endif
-#ifndef PAMM_CS_CTAS_PER_SM
-#define PAMM_CS_CTAS_PER_SM 2
-#endif
-constexpr int CS_CTAS_PER_SM = PAMM_CS_CTAS_PER_SM;       // the ring budget is per CTA
-constexpr int CS_MAX_CONSUMERS = PAMM_CS_MAX_CONSUMERS;   // consumer threads
-#ifndef PAMM_CS_MIN_VPT
-#define PAMM_CS_MIN_VPT 1
-#endif
-constexpr int CS_MIN_VPT = PAMM_CS_MIN_VPT;
+constexpr int CS_CTAS_PER_SM = 2;                // the ring budget is per CTA
+constexpr int CS_MAX_CONSUMERS = 384;            // consumer threads
+constexpr int CS_MIN_VPT = 1;
 constexpr int CS_MAX_VPT = 4;                    // 16-byte chunks per consumer thread
 constexpr int CS_MAX_SLOTS = 32;
-#ifndef PAMM_CS_MAX_RPS
-#define PAMM_CS_MAX_RPS 4
-#endif
-constexpr int CS_MAX_RPS = PAMM_CS_MAX_RPS;      // rows per ring slot, at most
+constexpr int CS_MAX_RPS = 4;                    // rows per ring slot, at most
 constexpr int CS_SLOT_TARGET_BYTES = 16 * 1024;  // rows are grouped while the slot stays within this
 constexpr uint32_t CS_PRODUCER_SPINS = 1u << 22;  // idle polls before the producer gives up
-constexpr int CS_RING_BYTES = PAMM_CS_RING_KB * 1024;
+constexpr int CS_RING_BYTES = 88 * 1024;
 
 struct ContractStreamPlan {
     int consumers;      // consumer threads, a multiple of 32
@@ -87,8 +72,8 @@ inline ContractStreamPlan contract_stream_plan(int64_t m, size_t esz) {
 
 template <typename T, int VPT, int RPS>
 __global__ void __launch_bounds__(CS_MAX_CONSUMERS + 32, CS_CTAS_PER_SM)
-contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ alpha, const T* __restrict__ dY,
-                       int64_t ldy, int64_t m, int k, const int32_t* __restrict__ seg_start,
+contract_stream_kernel(const void* __restrict__ f, int f_type, const float* __restrict__ alpha, const T* __restrict__ dY,
+                       int64_t ldy, int64_t b, int64_t m, int k, const int32_t* __restrict__ seg_start,
                        const int32_t* __restrict__ perm, int rows_per_cta, int slots, int row_pitch,
                        uint32_t bulk_bytes, float* __restrict__ partials, int64_t m_pad,
                        float* __restrict__ Bt, int64_t ldb) {
@@ -117,7 +102,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
     grid_dependency_wait();       // seg_start and perm come from the kernel before
     grid_launch_dependents();
 
-    const int32_t total = seg_start[k];
+    const int32_t total = (int32_t)min((int64_t)max(seg_start[k], 0), b);     // = b unless some f_i were out of range
     const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
     const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
     const int nrows = r_end - r_begin;
@@ -133,15 +118,28 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
         int32_t r = lane < slots ? r_begin + lane * RPS : r_end;     // first sorted position of my next slot load
         int32_t i_cur[RPS], i_nxt[RPS], j_cur[RPS];
         float a_cur[RPS];
+        // A sorted position holds a row id in [0, b) unless the sort was fed counts that do not
+        // belong to this f; such an entry is reported and replaced by row 0 with weight zero.
+        bool bad_perm = false;
+        auto row_at = [&](int32_t pos) {
+            int32_t i = perm[pos];
+            if ((uint32_t)i >= (uint32_t)b) { bad_perm = true; i = -1; }
+            return i;
+        };
+        auto weight_of = [&](int32_t i) { return i >= 0 ? alpha[i] : 0.f; };
+        auto segment_of_row = [&](int32_t i) {
+            const int32_t j = i >= 0 ? load_index(f, f_type, i) : 0;
+            return min(max(j, 0), k - 1);
+        };
 #pragma unroll
         for (int u = 0; u < RPS; ++u) {
             i_cur[u] = -1; i_nxt[u] = -1; j_cur[u] = 0; a_cur[u] = 0.f;
             if (r + u < r_end) {
-                i_cur[u] = perm[r + u];
-                a_cur[u] = alpha[i_cur[u]];
-                j_cur[u] = f[i_cur[u]];
+                i_cur[u] = row_at(r + u);
+                a_cur[u] = weight_of(i_cur[u]);
+                j_cur[u] = segment_of_row(i_cur[u]);
             }
-            if (r + round_rows + u < r_end) i_nxt[u] = perm[r + round_rows + u];
+            if (r + round_rows + u < r_end) i_nxt[u] = row_at(r + round_rows + u);
         }
         const uint64_t stream_policy = ptx::l2_policy_evict_first();   // dY is read once
         uint32_t phase = 0, idle = 0;
@@ -159,7 +157,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                     for (int u = 0; u < RPS; ++u)
                         if (u < valid)
                             ptx::bulk_load_hint(ring + (size_t)lane * slot_bytes + (size_t)u * row_pitch,
-                                                dY + (int64_t)i_cur[u] * ldy, bulk_bytes, &s_full[lane], stream_policy);
+                                                dY + (int64_t)max(i_cur[u], 0) * ldy, bulk_bytes, &s_full[lane], stream_policy);
                 } else {
                     ptx::mbar_arrive(&s_full[lane]);
                 }
@@ -171,10 +169,10 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                 for (int u = 0; u < RPS; ++u) {
                     i_cur[u] = i_nxt[u];
                     if (r + u < r_end) {
-                        a_cur[u] = alpha[i_cur[u]];
-                        j_cur[u] = f[i_cur[u]];
+                        a_cur[u] = weight_of(i_cur[u]);
+                        j_cur[u] = segment_of_row(i_cur[u]);
                     }
-                    i_nxt[u] = r + round_rows + u < r_end ? perm[r + round_rows + u] : -1;
+                    i_nxt[u] = r + round_rows + u < r_end ? row_at(r + round_rows + u) : -1;
                 }
                 progressed = true;
             }
@@ -185,6 +183,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                 __nanosleep(32);
             }
         }
+        if (bad_perm) raise_status(DEV_BAD_INDEX);
         if (!ok) {
             if (lane == 0) {
                 *abort_flag = 1;
@@ -275,7 +274,7 @@ contract_stream_kernel(const int32_t* __restrict__ f, const float* __restrict__ 
                             fma_raw<T>(acc[v], a, raw[u][v]);
                         } else if (vec < nvec) {     // the ragged last chunk of the row comes straight from global memory
                             float x[V];
-                            load_vec<T>(dY + (int64_t)row * ldy, vec * V, m, x);
+                            load_vec<T>(dY + (int64_t)max(row, 0) * ldy, vec * V, m, x);
 #pragma unroll
                             for (int e = 0; e < V; ++e) acc[v][e] = fmaf(a, x[e], acc[v][e]);
                         }

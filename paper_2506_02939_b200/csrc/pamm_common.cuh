@@ -26,8 +26,30 @@ __device__ __forceinline__ void raise_status(int bit) { atomicOr(&g_status_word,
 // returns once the predecessor has finished and its writes are visible, and is
 // a no-op for an ordinary launch.  grid_launch_dependents() lets the successor's
 // CTAs be scheduled as soon as every CTA of this grid has issued it.
+//
+// RULE for every kernel of this library: call grid_dependency_wait() before the first
+// access to global memory that a predecessor may write (or may still read, if this kernel
+// overwrites it).  Kernels rely on it transitively: a kernel may release its dependents
+// before its own wait has returned (the tensor-core compress kernel does, so that its
+// successor's set-up overlaps the whole pass), and the successor's wait then still covers
+// everything older, because it returns only when the predecessor grid -- which itself
+// waited for its own predecessor -- has completed.  A kernel that reads anything before its
+// wait may read only what was complete before its predecessor was LAUNCHED.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ---- the assignment f in its storage type ------------------------------------------
+// `type` is a pamm_index_type: 32-bit signed, or unsigned 16 / 8 bits for k <= 65536 / 256.
+__device__ __forceinline__ void store_index(void* f, int type, int64_t i, int32_t j) {
+    if (type == PAMM_IDX_I32) static_cast<int32_t*>(f)[i] = j;
+    else if (type == PAMM_IDX_U16) static_cast<uint16_t*>(f)[i] = (uint16_t)j;
+    else static_cast<uint8_t*>(f)[i] = (uint8_t)j;
+}
+__device__ __forceinline__ int32_t load_index(const void* f, int type, int64_t i) {
+    if (type == PAMM_IDX_I32) return static_cast<const int32_t*>(f)[i];
+    if (type == PAMM_IDX_U16) return (int32_t)static_cast<const uint16_t*>(f)[i];
+    return (int32_t)static_cast<const uint8_t*>(f)[i];
+}
 
 // Normalisation factor of Section 3.2 ("Normalization factor beta", Eq. 4-5):
 // beta = b / (b - eta) with eta dropped rows, read from device memory; 1 when no
@@ -139,6 +161,21 @@ __host__ __device__ inline uint32_t perm_apply(const PermKey& pk, uint32_t x) {
 }
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Text behind the last PAMM_ERR_CUDA of the calling thread (which CUDA call failed and how).
+void note_cuda_failure(const char* what, cudaError_t err);
+// cudaGetLastError as a status, with the failure noted.
+inline pamm_status launch_result(const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return PAMM_OK;
+    note_cuda_failure(what, e);
+    return PAMM_ERR_CUDA;
+}
+
+inline pamm_status tensor_map_failed() {
+    note_cuda_failure("cuTensorMapEncodeTiled (tensor map of an operand)", cudaErrorInvalidValue);
+    return PAMM_ERR_CUDA;
+}
 
 // Raises a kernel's dynamic shared-memory limit when a launch needs more than the
 // 48 KiB default, remembering per device and kernel what has been granted already

@@ -22,6 +22,11 @@
 using namespace pamm;
 
 namespace pamm {
+static thread_local char g_cuda_detail[256] = "";
+void note_cuda_failure(const char* what, cudaError_t err) {
+    snprintf(g_cuda_detail, sizeof g_cuda_detail, "%s: %s (%s)", what, cudaGetErrorName(err), cudaGetErrorString(err));
+}
+
 bool ensure_dynamic_smem(const void* kernel, size_t bytes) {
     if (bytes <= 48 * 1024) return true;
     static std::mutex mu;
@@ -31,7 +36,12 @@ bool ensure_dynamic_smem(const void* kernel, size_t bytes) {
     std::lock_guard<std::mutex> lock(mu);
     size_t& have = granted[{dev, kernel}];
     if (have >= bytes) return true;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return false;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) {
+        note_cuda_failure("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+        cudaGetLastError();
+        return false;
+    }
     have = bytes;
     return true;
 }
@@ -41,9 +51,13 @@ namespace {
 
 inline size_t esize(pamm_dtype dt) { return dt == PAMM_BF16 ? 2 : 4; }
 inline bool dtype_ok(pamm_dtype dt) { return dt == PAMM_F32 || dt == PAMM_BF16; }
+inline bool layout_ok(pamm_layout l) { return l == PAMM_DW_NM || l == PAMM_DW_MN; }
+inline bool index_type_ok(pamm_index_type t) { return t == PAMM_IDX_I32 || t == PAMM_IDX_U16 || t == PAMM_IDX_U8; }
+inline size_t index_size(pamm_index_type t) { return t == PAMM_IDX_I32 ? 4 : t == PAMM_IDX_U16 ? 2 : 1; }
+inline int64_t index_limit(pamm_index_type t) { return t == PAMM_IDX_I32 ? (1ll << 31) - 1 : t == PAMM_IDX_U16 ? 65536 : 256; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline bool ld_ok(int64_t ld, int64_t cols, size_t es) { return ld >= cols && (ld * (int64_t)es) % 16 == 0; }
-inline pamm_status launch_status() { return cudaGetLastError() == cudaSuccess ? PAMM_OK : PAMM_ERR_CUDA; }
+inline pamm_status launch_status() { return launch_result("kernel launch"); }
 constexpr int64_t MAX_ROWS = (1ll << 31) - 1024;   // row ids, counts and offsets are int32
 
 // Kernel launches issued so far (all streams), and optional event pairs that
@@ -72,8 +86,30 @@ inline void launch(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaS
     g_launches += 1;
 }
 
+int sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            sms = 148;
+    }
+    return sms;
+}
+
+// The row partition shared by the compress pass and the counting sort of the backward pass.
+inline int64_t sort_rows_per_block(int64_t b) { return compress_rows_per_cta(b, sm_count()); }
+inline ContractWs contract_ws(void* base, int64_t b, int64_t m, int64_t k) {
+    return contract_ws_layout(base, b, m, k, sort_rows_per_block(b));
+}
+// Bytes of the per-block histograms of f for one generator set (the "sort products").
+inline size_t sort_products_bytes(int64_t b, int64_t k) {
+    const int64_t rpb = sort_rows_per_block(b);
+    return (size_t)round_up(((b + rpb - 1) / rpb) * k * 4, 256);
+}
+
 struct StepArena {
-    char *X, *dY, *C, *dW, *Bt, *ws;
+    char *X, *dY, *C, *dW, *Bt, *ws, *products;
     float *invnorm, *alpha;
     int32_t *idx, *f;
     int64_t ldx, ldy, ldc, ldw, ldb;
@@ -98,8 +134,9 @@ StepArena step_arena_layout(void* base, int64_t b, int64_t n, int64_t m, int64_t
     a.alpha = (float*)take((size_t)b * 4);
     a.Bt = take((size_t)k * a.ldb * 4);
     a.dW = take((size_t)n * a.ldw * 4);
-    a.ws_bytes = contract_ws_layout(nullptr, b, m, k).bytes;
+    a.ws_bytes = contract_ws(nullptr, b, m, k).bytes;
     a.ws = take(a.ws_bytes);
+    a.products = take(sort_products_bytes(b, k));
     a.bytes = off;
     return a;
 }
@@ -128,8 +165,8 @@ constexpr Neighbourhood NO_NEIGHBOURHOOD = {false, 0.f, nullptr};
 
 template <typename T>
 pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,
-                                 int64_t k, const float* c_invnorm, int32_t* f, float* alpha, const Neighbourhood& nb,
-                                 cudaStream_t st) {
+                                 int64_t k, const float* c_invnorm, void* f, int f_type, float* alpha,
+                                 const Neighbourhood& nb, cudaStream_t st) {
     const int64_t want = (b + CS_WARPS - 1) / CS_WARPS;
     const int grid = (int)std::min<int64_t>(want, 148 * 8);
     const float eps2 = nb.eps * nb.eps, slack = neighbourhood_slack(n);
@@ -137,7 +174,7 @@ pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t 
                       : (k <= 4 ? compress_simt_kernel<T, 4, false> : compress_simt_kernel<T, 8, false>);
     prof_begin(PAMM_PROF_COMPRESS, st);
     launch(kern, dim3(grid), dim3(CS_THREADS), 0, st, true, (const T*)X, ldx, b, n, (const T*)C, ldc, (int)k, c_invnorm, f,
-           alpha, eps2, slack, nb.dropped);
+           f_type, alpha, eps2, slack, nb.dropped);
     prof_end(PAMM_PROF_COMPRESS, st);
     return launch_status();
 }
@@ -146,37 +183,46 @@ pamm_status launch_compress_simt(const void* X, int64_t ldx, int64_t b, int64_t 
 // which every block rebuilds the scan on its own instead of a separate launch.
 constexpr int64_t FUSED_SCAN_LIMIT = 1ll << 24;
 
-int sm_count() {
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
-            sms = 148;
-    }
-    return sms;
-}
-
-template <typename T>
-pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
-                            int64_t k, float* Bt, int64_t ldb, const ContractWs& w, cudaStream_t st) {
-    constexpr int V = Vec16<T>::N;
+// The counting sort of the rows by f.  `products` (the per-block histograms the compress
+// pass left behind) saves the histogram launch.
+pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const int32_t* products, const ContractWs& w,
+                        cudaStream_t st) {
     const size_t hsmem = (size_t)k * 4;
     if (!ensure_dynamic_smem((const void*)contract_hist_kernel, hsmem) ||
         !ensure_dynamic_smem((const void*)contract_scatter_kernel, hsmem) ||
         !ensure_dynamic_smem((const void*)contract_scan_scatter_kernel, hsmem))
         return PAMM_ERR_CUDA;
-    launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k, w.hist);
-    if (w.nb * w.nb * k <= FUSED_SCAN_LIMIT) {
-        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
-               (const int32_t*)w.hist, (int)w.nb, w.seg_start, w.perm);
+    const int rpb = (int)w.rows_per_block;
+    const bool fused_scan = w.nb * w.nb * k <= FUSED_SCAN_LIMIT;
+    const int32_t* hist = w.hist;
+    if (products && fused_scan) {
+        hist = products;            // read in place
+    } else if (products) {          // the scan below rewrites the table: work on a copy
+        if (cudaMemcpyAsync(w.hist, products, (size_t)w.nb * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return PAMM_ERR_CUDA;
+    } else {
+        launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb, w.hist);
+    }
+    if (fused_scan) {
+        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb,
+               hist, (int)w.nb, w.seg_start, w.perm);
     } else {
         launch(contract_scan_kernel, dim3(1), dim3(SCAN_THREADS), 0, st, true, w.hist, (int)w.nb, (int)k, w.seg_start);
-        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, b, (int)k,
+        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb,
                (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
     }
+    return launch_status();
+}
+
+template <typename T>
+pamm_status launch_contract(const void* f, int f_type, const float* alpha, const void* dY, int64_t ldy, int64_t b,
+                            int64_t m, int64_t k, float* Bt, int64_t ldb, const int32_t* products, const ContractWs& w,
+                            cudaStream_t st) {
+    constexpr int V = Vec16<T>::N;
+    pamm_status s = launch_sort(f, f_type, b, k, products, w, st);
+    if (s != PAMM_OK) return s;
     if (contract_stream_supported(m, sizeof(T))) {
-        // one balanced wave, one CTA per SM: rows of dY stream through a shared-memory ring
+        // one balanced wave, two CTAs per SM: rows of dY stream through a shared-memory ring
         const ContractStreamPlan p = contract_stream_plan(m, sizeof(T));
         int64_t ranges = std::min<int64_t>(CT_MAX_CTAS, (int64_t)sm_count() * CS_CTAS_PER_SM);
         const int64_t rows_per_cta = std::max<int64_t>(32, (b + ranges - 1) / ranges);
@@ -188,13 +234,13 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
                                  : contract_stream_kernel<T, 1, 1>;
         if (!ensure_dynamic_smem((const void*)kern, p.smem_bytes)) return PAMM_ERR_CUDA;
         prof_begin(PAMM_PROF_CONTRACT, st);
-        launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, alpha, (const T*)dY, ldy, m,
-               (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots, p.row_pitch,
-               p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
+        launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, f_type, alpha, (const T*)dY,
+               ldy, b, m, (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots,
+               p.row_pitch, p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
         prof_end(PAMM_PROF_CONTRACT, st);
         const int64_t items = k * (w.m_pad / 4);
         launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st,
-               true, (const float*)w.partials, w.m_pad, m, (int)k, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
+               true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
         return launch_status();
     }
     // very wide rows: column slabs, register staging
@@ -209,23 +255,41 @@ pamm_status launch_contract(const int32_t* f, const float* alpha, const void* dY
     ranges = (b + rows_per_cta - 1) / rows_per_cta;
     dim3 grid((unsigned)ranges, (unsigned)slabs);
     prof_begin(PAMM_PROF_CONTRACT, st);
-    launch(contract_main_kernel<T>, grid, dim3(threads), 0, st, true, alpha, (const T*)dY, ldy, m, (int)k,
+    launch(contract_main_kernel<T>, grid, dim3(threads), 0, st, true, alpha, (const T*)dY, ldy, b, m, (int)k,
            (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, w.partials, w.m_pad, Bt, ldb);
     prof_end(PAMM_PROF_CONTRACT, st);
     const int64_t items = k * (w.m_pad / 4);
     launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st, true,
-           (const float*)w.partials, w.m_pad, m, (int)k, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
+           (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
     return launch_status();
 }
 
+// How the weight gradient is stored.
+struct DwSpec {
+    void* ptr;
+    int64_t ld;
+    pamm_dtype dt;
+    pamm_layout layout;
+};
+
 template <typename T>
 pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64_t n, const float* Bt, int64_t ldb,
-                                    int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows,
+                                    int64_t m, const DwSpec& dw, cudaStream_t st, int64_t b_rows,
                                     const int32_t* dropped, bool accumulate) {
-    const int64_t items = n * ((m + 3) / 4);
+    const bool swap = dw.layout == PAMM_DW_MN;
+    const int64_t rows = swap ? m : n, cols = swap ? n : m;
+    const int64_t items = rows * ((cols + 3) / 4);
+    const dim3 grid((unsigned)((items + WG_THREADS - 1) / WG_THREADS)), block(WG_THREADS);
     prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-    launch(weight_grad_simt_kernel<T>, dim3((unsigned)((items + WG_THREADS - 1) / WG_THREADS)), dim3(WG_THREADS), 0, st, true,
-           (const T*)C, ldc, (int)k, n, Bt, ldb, m, dW, ldw, b_rows, dropped, accumulate ? 1 : 0);
+    if (dw.dt == PAMM_F32) {
+        auto kern = swap ? weight_grad_simt_kernel<T, float, true> : weight_grad_simt_kernel<T, float, false>;
+        launch(kern, grid, block, 0, st, true, (const T*)C, ldc, (int)k, n, Bt, ldb, m, (float*)dw.ptr, dw.ld, b_rows, dropped,
+               accumulate ? 1 : 0);
+    } else {
+        auto kern = swap ? weight_grad_simt_kernel<T, __nv_bfloat16, true> : weight_grad_simt_kernel<T, __nv_bfloat16, false>;
+        launch(kern, grid, block, 0, st, true, (const T*)C, ldc, (int)k, n, Bt, ldb, m, (__nv_bfloat16*)dw.ptr, dw.ld, b_rows,
+               dropped, accumulate ? 1 : 0);
+    }
     prof_end(PAMM_PROF_WEIGHT_GRAD, st);
     return launch_status();
 }
@@ -241,81 +305,114 @@ pamm_status check_select(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_
     return PAMM_OK;
 }
 
+// The sort products are optional: no buffer, none written.
+pamm_status check_products_out(const void* ws, size_t ws_bytes, int64_t b, int64_t k, int groups) {
+    if (!ws) return PAMM_OK;
+    if (!aligned(ws, 256) || ws_bytes < (size_t)groups * sort_products_bytes(b, k)) return PAMM_ERR_WORKSPACE;
+    return PAMM_OK;
+}
+
 pamm_status check_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C,
-                           int64_t ldc, int64_t k, const float* c_invnorm, int32_t* f, float* alpha) {
-    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+                           int64_t ldc, int64_t k, const float* c_invnorm, void* f, pamm_index_type f_type, float* alpha) {
+    if (!dtype_ok(dt) || !index_type_ok(f_type)) return PAMM_ERR_UNSUPPORTED;
     if (!X || !C || !c_invnorm || !f || !alpha) return PAMM_ERR_INVALID_ARG;
     if (b < 1 || n < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (k > index_limit(f_type)) return PAMM_ERR_INVALID_ARG;     // f_i would not fit its storage type
     if (!ld_ok(ldx, n, esize(dt)) || !ld_ok(ldc, n, esize(dt))) return PAMM_ERR_INVALID_ARG;
-    if (!aligned(X, 16) || !aligned(C, 16) || !aligned(f, 4) || !aligned(alpha, 4) || !aligned(c_invnorm, 4))
+    if (!aligned(X, 16) || !aligned(C, 16) || !aligned(f, index_size(f_type)) || !aligned(alpha, 4) || !aligned(c_invnorm, 4))
         return PAMM_ERR_INVALID_ARG;
     return PAMM_OK;
 }
 
-pamm_status check_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
-                           pamm_dtype dt, int64_t k, const float* Bt, int64_t ldb, bool bt_required,
-                           const void* ws, size_t ws_bytes) {
-    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+pamm_status check_contract(const void* f, pamm_index_type f_type, const float* alpha, const void* dY, int64_t ldy,
+                           int64_t b, int64_t m, pamm_dtype dt, int64_t k, const float* Bt, int64_t ldb, bool bt_required,
+                           const void* products, const void* ws, size_t ws_bytes) {
+    if (!dtype_ok(dt) || !index_type_ok(f_type)) return PAMM_ERR_UNSUPPORTED;
     if (!f || !alpha || !dY || (bt_required && !Bt)) return PAMM_ERR_INVALID_ARG;
     if (b < 1 || m < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (k > index_limit(f_type)) return PAMM_ERR_INVALID_ARG;
     if (!ld_ok(ldy, m, esize(dt)) || (Bt && !ld_ok(ldb, m, 4))) return PAMM_ERR_INVALID_ARG;
-    if (!aligned(dY, 16) || (Bt && !aligned(Bt, 16)) || !aligned(f, 4) || !aligned(alpha, 4)) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(dY, 16) || (Bt && !aligned(Bt, 16)) || !aligned(f, index_size(f_type)) || !aligned(alpha, 4))
+        return PAMM_ERR_INVALID_ARG;
+    if (products && !aligned(products, 256)) return PAMM_ERR_INVALID_ARG;
     if (k > CT_MAX_K) return PAMM_ERR_UNSUPPORTED;
     if (!ws || !aligned(ws, 256)) return PAMM_ERR_WORKSPACE;
-    if (ws_bytes < contract_ws_layout(nullptr, b, m, k).bytes) return PAMM_ERR_WORKSPACE;
+    if (ws_bytes < contract_ws(nullptr, b, m, k).bytes) return PAMM_ERR_WORKSPACE;
     return PAMM_OK;
 }
 
 pamm_status check_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
-                              int64_t ldb, int64_t m, float* dW, int64_t ldw) {
-    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
-    if (!C || !Bt || !dW) return PAMM_ERR_INVALID_ARG;
+                              int64_t ldb, int64_t m, const DwSpec& dw) {
+    if (!dtype_ok(dt) || !dtype_ok(dw.dt) || !layout_ok(dw.layout)) return PAMM_ERR_UNSUPPORTED;
+    if (!C || !Bt || !dw.ptr) return PAMM_ERR_INVALID_ARG;
     if (k < 1 || n < 1 || m < 1) return PAMM_ERR_INVALID_ARG;
-    if (!ld_ok(ldc, n, esize(dt)) || !ld_ok(ldb, m, 4) || !ld_ok(ldw, m, 4)) return PAMM_ERR_INVALID_ARG;
-    if (!aligned(C, 16) || !aligned(Bt, 16) || !aligned(dW, 16)) return PAMM_ERR_INVALID_ARG;
+    const int64_t out_cols = dw.layout == PAMM_DW_MN ? n : m;
+    if (!ld_ok(ldc, n, esize(dt)) || !ld_ok(ldb, m, 4) || !ld_ok(dw.ld, out_cols, esize(dw.dt))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(C, 16) || !aligned(Bt, 16) || !aligned(dw.ptr, 16)) return PAMM_ERR_INVALID_ARG;
     return PAMM_OK;
 }
 
 // x_is_ready: X was complete before the previous kernel of the stream started (true
 // after our own select kernel), so the compress kernel may read it before that
-// kernel has finished.
+// kernel has finished.  `groups` generator sets are served by one pass over X where the
+// tensor-core kernel applies, else by one CUDA-core pass per set.  `products` (optional)
+// receives the per-block histograms of f.
 pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
-                        int64_t k, const float* c_invnorm, int32_t* f, float* alpha, bool x_is_ready, cudaStream_t st,
+                        int64_t k, int groups, const float* c_invnorm, void* f, pamm_index_type f_type, float* alpha,
+                        int64_t out_stride, int32_t* products, bool x_is_ready, cudaStream_t st,
                         const Neighbourhood& nb = NO_NEIGHBOURHOOD) {
-    if (dt == PAMM_F32) return launch_compress_simt<float>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, nb, st);
-    if (compress_umma_supported(b, n, k)) {
+    if (dt == PAMM_BF16 && compress_umma_usable(b, n, k, groups, sm_count(), nb.on)) {
+        const CompressOut out = {f, alpha, out_stride, products, (int64_t)(sort_products_bytes(b, k) / 4), (int)f_type};
         prof_begin(PAMM_PROF_COMPRESS, st);
-        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, sm_count(), x_is_ready, st,
+        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, groups, c_invnorm, out, sm_count(), x_is_ready, st,
                                                     nb.on, nb.eps, nb.dropped);
         prof_end(PAMM_PROF_COMPRESS, st);
         g_launches += 1;
         return s;
     }
-    return launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, C, ldc, k, c_invnorm, f, alpha, nb, st);
+    const size_t es = esize(dt), fs = index_size(f_type);
+    const int64_t rpb = sort_rows_per_block(b), nblk = (b + rpb - 1) / rpb;
+    if (products && !ensure_dynamic_smem((const void*)contract_hist_kernel, (size_t)k * 4)) return PAMM_ERR_CUDA;
+    for (int g = 0; g < groups; ++g) {
+        const char* Cg = (const char*)C + (size_t)g * k * ldc * es;
+        void* fg = (char*)f + (size_t)g * out_stride * fs;
+        float* ag = alpha + (size_t)g * out_stride;
+        const pamm_status s = dt == PAMM_F32
+            ? launch_compress_simt<float>(X, ldx, b, n, Cg, ldc, k, c_invnorm + (size_t)g * 2 * k, fg, (int)f_type, ag, nb, st)
+            : launch_compress_simt<__nv_bfloat16>(X, ldx, b, n, Cg, ldc, k, c_invnorm + (size_t)g * 2 * k, fg, (int)f_type, ag, nb, st);
+        if (s != PAMM_OK) return s;
+        if (products)
+            launch(contract_hist_kernel, dim3((unsigned)nblk), dim3(SORT_BLK), (size_t)k * 4, st, true, (const void*)fg,
+                   (int)f_type, b, (int)k, (int)rpb, products + (size_t)g * (sort_products_bytes(b, k) / 4));
+    }
+    return launch_status();
 }
 
 pamm_status do_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Bt,
-                           int64_t ldb, int64_t m, float* dW, int64_t ldw, cudaStream_t st, int64_t b_rows = 0,
+                           int64_t ldb, int64_t m, const DwSpec& dw, cudaStream_t st, int64_t b_rows = 0,
                            const int32_t* dropped = nullptr, bool accumulate = false) {
     if (dt == PAMM_F32)
-        return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
-    if (weight_grad_persist_supported(k, n, m)) {
+        return launch_weight_grad_simt<float>(C, ldc, k, n, Bt, ldb, m, dw, st, b_rows, dropped, accumulate);
+    const bool bf16_out = dw.dt == PAMM_BF16, swap = dw.layout == PAMM_DW_MN;
+    // the TMA stores need at least one whole 16-byte unit per output row
+    const bool tma_ok = (swap ? n : m) * (int64_t)esize(dw.dt) >= 16;
+    if (tma_ok && weight_grad_persist_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped,
-                                                          accumulate);
+        const pamm_status s = launch_weight_grad_persist(C, ldc, k, n, Bt, ldb, m, dw.ptr, dw.ld, bf16_out, swap, sm_count(), st,
+                                                          b_rows, dropped, accumulate);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
-    if (weight_grad_chunked_supported(k, n, m)) {
+    if (tma_ok && weight_grad_chunked_supported(k, n, m)) {
         prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
-        const pamm_status s = launch_weight_grad_chunked(C, ldc, k, n, Bt, ldb, m, dW, ldw, sm_count(), st, b_rows, dropped,
-                                                         accumulate);
+        const pamm_status s = launch_weight_grad_chunked(C, ldc, k, n, Bt, ldb, m, dw.ptr, dw.ld, bf16_out, swap, sm_count(), st,
+                                                         b_rows, dropped, accumulate);
         prof_end(PAMM_PROF_WEIGHT_GRAD, st);
         g_launches += 1;
         return s;
     }
-    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dW, ldw, st, b_rows, dropped, accumulate);
+    return launch_weight_grad_simt<__nv_bfloat16>(C, ldc, k, n, Bt, ldb, m, dw, st, b_rows, dropped, accumulate);
 }
 
 }  // namespace
@@ -357,7 +454,9 @@ const char* pamm_status_string(pamm_status s) {
     return "unknown status";
 }
 
-int pamm_version(void) { return 100; }
+int pamm_version(void) { return 200; }
+
+const char* pamm_last_error_detail(void) { return g_cuda_detail; }
 
 unsigned long long pamm_launch_count(void) { return g_launches; }
 
@@ -373,15 +472,26 @@ size_t pamm_workspace_bytes(pamm_ws_kind kind, int64_t b, int64_t n, int64_t m, 
     switch (kind) {
         case PAMM_WS_COMPRESS:
             if (n < 1) return (size_t)-1;
-            return 0;
+            return sort_products_bytes(b, k);
         case PAMM_WS_CONTRACT:
             if (m < 1) return (size_t)-1;
-            return contract_ws_layout(nullptr, b, m, k).bytes;
+            return contract_ws(nullptr, b, m, k).bytes;
         case PAMM_WS_STEP_HOST:
             if (n < 1 || m < 1) return (size_t)-1;
             return step_arena_layout(nullptr, b, n, m, k, dt).bytes;
     }
     return (size_t)-1;
+}
+
+pamm_status pamm_saved_bytes(int64_t b, int64_t n, int64_t k, pamm_dtype dt, pamm_index_type f_type, int64_t out[4]) {
+    if (!dtype_ok(dt) || !index_type_ok(f_type)) return PAMM_ERR_UNSUPPORTED;
+    if (!out || b < 1 || n < 1 || k < 1 || k > b || k > index_limit(f_type)) return PAMM_ERR_INVALID_ARG;
+    const int64_t e = (int64_t)esize(dt);
+    out[0] = b * n * e;                                             // X itself
+    out[1] = k * n * e + b * (int64_t)index_size(f_type) + b * 4;   // C, f, alpha
+    out[2] = b * n;                                                 // scalars, as the paper counts them
+    out[3] = k * n + 2 * b;
+    return PAMM_OK;
 }
 
 pamm_status pamm_draw_indices_host(int64_t b, int64_t k, uint64_t seed, int32_t* idx_out) {
@@ -403,94 +513,122 @@ pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_
 }
 
 pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C, int64_t ldc,
-                          int64_t k, const float* c_invnorm, int32_t* f, float* alpha, void* workspace,
-                          size_t ws_bytes, void* stream) {
-    (void)workspace; (void)ws_bytes;
-    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+                          int64_t k, const float* c_invnorm, void* f, pamm_index_type f_type, float* alpha,
+                          void* workspace, size_t ws_bytes, void* stream) {
+    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, f_type, alpha);
     if (s != PAMM_OK) return s;
-    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, false, (cudaStream_t)stream);
+    s = check_products_out(workspace, ws_bytes, b, k, 1);
+    if (s != PAMM_OK) return s;
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, 1, c_invnorm, f, f_type, alpha, b, (int32_t*)workspace, false,
+                       (cudaStream_t)stream);
+}
+
+pamm_status pamm_compress_projections(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C,
+                                      int64_t ldc, int64_t k, int64_t sets, const float* c_invnorm, void* f,
+                                      pamm_index_type f_type, float* alpha, int64_t out_stride, void* workspace,
+                                      size_t ws_bytes, void* stream) {
+    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, f_type, alpha);
+    if (s != PAMM_OK) return s;
+    if (sets < 1 || sets > 64 || out_stride < b || (out_stride * (int64_t)index_size(f_type)) % 4) return PAMM_ERR_INVALID_ARG;
+    s = check_products_out(workspace, ws_bytes, b, k, (int)sets);
+    if (s != PAMM_OK) return s;
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, (int)sets, c_invnorm, f, f_type, alpha, out_stride, (int32_t*)workspace,
+                       false, (cudaStream_t)stream);
 }
 
 pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, int64_t k,
                                 uint64_t seed, const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc,
-                                float* c_invnorm, int32_t* f, float* alpha, void* workspace, size_t ws_bytes,
-                                void* stream) {
-    (void)workspace; (void)ws_bytes;
+                                float* c_invnorm, void* f, pamm_index_type f_type, float* alpha, void* workspace,
+                                size_t ws_bytes, void* stream) {
     pamm_status s = check_select(X, ldx, b, n, dt, k, idx_out, C, ldc, c_invnorm);
     if (s != PAMM_OK) return s;
-    s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+    s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, f_type, alpha);
+    if (s != PAMM_OK) return s;
+    s = check_products_out(workspace, ws_bytes, b, k, 1);
     if (s != PAMM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     s = dt == PAMM_F32 ? launch_select<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st)
                        : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
     if (s != PAMM_OK) return s;
-    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, true, st);
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, 1, c_invnorm, f, f_type, alpha, b, (int32_t*)workspace, true, st);
 }
 
-pamm_status pamm_contract(const int32_t* f, const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
-                          pamm_dtype dt, int64_t k, float* Btilde, int64_t ldb, void* workspace, size_t ws_bytes,
-                          void* stream) {
-    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, workspace, ws_bytes);
+pamm_status pamm_contract(const void* f, pamm_index_type f_type, const float* alpha, const void* dY, int64_t ldy,
+                          int64_t b, int64_t m, pamm_dtype dt, int64_t k, float* Btilde, int64_t ldb,
+                          const void* sort_products, void* workspace, size_t ws_bytes, void* stream) {
+    pamm_status s = check_contract(f, f_type, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, sort_products, workspace, ws_bytes);
     if (s != PAMM_OK) return s;
-    const ContractWs w = contract_ws_layout(workspace, b, m, k);
+    const ContractWs w = contract_ws(workspace, b, m, k);
     cudaStream_t st = (cudaStream_t)stream;
-    return dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st)
-                          : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st);
+    const int32_t* pr = (const int32_t*)sort_products;
+    return dt == PAMM_F32 ? launch_contract<float>(f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, pr, w, st)
+                          : launch_contract<__nv_bfloat16>(f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, pr, w, st);
 }
 
 pamm_status pamm_weight_grad(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Btilde,
-                             int64_t ldb, int64_t m, float* dW, int64_t ldw, void* stream) {
-    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+                             int64_t ldb, int64_t m, void* dW, int64_t ldw, pamm_dtype dw_dt, pamm_layout layout,
+                             void* stream) {
+    const DwSpec dw = {dW, ldw, dw_dt, layout};
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw);
     if (s != PAMM_OK) return s;
-    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream);
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw, (cudaStream_t)stream);
 }
 
 pamm_status pamm_compress_eps(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt, const void* C,
-                              int64_t ldc, int64_t k, const float* c_invnorm, float eps, int32_t* f, float* alpha,
-                              int32_t* dropped, void* workspace, size_t ws_bytes, void* stream) {
-    (void)workspace; (void)ws_bytes;
-    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha);
+                              int64_t ldc, int64_t k, const float* c_invnorm, float eps, void* f,
+                              pamm_index_type f_type, float* alpha, int32_t* dropped, void* workspace, size_t ws_bytes,
+                              void* stream) {
+    pamm_status s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, f_type, alpha);
     if (s != PAMM_OK) return s;
     if (!dropped || !aligned(dropped, 4) || !(eps >= 0.f)) return PAMM_ERR_INVALID_ARG;     // also rejects NaN
+    s = check_products_out(workspace, ws_bytes, b, k, 1);
+    if (s != PAMM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(dropped, 0, sizeof(int32_t), st) != cudaSuccess) return PAMM_ERR_CUDA;
     // ||X_i - alpha C_f|| <= ||X_i|| always, so eps >= 1 keeps every row: the plain kernel does
     const bool on = eps < 1.f;
-    return do_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, alpha, false, st, Neighbourhood{on, eps, dropped});
+    return do_compress(X, ldx, b, n, dt, C, ldc, k, 1, c_invnorm, f, f_type, alpha, b, (int32_t*)workspace, false, st,
+                       Neighbourhood{on, eps, dropped});
 }
 
 pamm_status pamm_weight_grad_beta(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt, const float* Btilde,
-                                  int64_t ldb, int64_t m, int64_t b, const int32_t* dropped, float* dW, int64_t ldw,
-                                  void* stream) {
-    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+                                  int64_t ldb, int64_t m, int64_t b, const int32_t* dropped, void* dW, int64_t ldw,
+                                  pamm_dtype dw_dt, pamm_layout layout, void* stream) {
+    const DwSpec dw = {dW, ldw, dw_dt, layout};
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw);
     if (s != PAMM_OK) return s;
     if (b < 1 || (dropped && !aligned(dropped, 4))) return PAMM_ERR_INVALID_ARG;
-    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream, b, dropped);
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw, (cudaStream_t)stream, b, dropped);
 }
 
 pamm_status pamm_weight_grad_accumulate(const void* C, int64_t ldc, int64_t k, int64_t n, pamm_dtype dt,
-                                        const float* Btilde, int64_t ldb, int64_t m, float* dW, int64_t ldw, void* stream) {
-    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw);
+                                        const float* Btilde, int64_t ldb, int64_t m, float* dW, int64_t ldw,
+                                        pamm_layout layout, void* stream) {
+    const DwSpec dw = {dW, ldw, PAMM_F32, layout};
+    pamm_status s = check_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw);
     if (s != PAMM_OK) return s;
-    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dW, ldw, (cudaStream_t)stream, 0, nullptr, true);
+    return do_weight_grad(C, ldc, k, n, dt, Btilde, ldb, m, dw, (cudaStream_t)stream, 0, nullptr, true);
 }
 
-pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, const int32_t* f, const float* alpha,
-                                      const void* dY, int64_t ldy, int64_t b, int64_t m, pamm_dtype dt, int64_t k,
-                                      float* Btilde, int64_t ldb, float* dW, int64_t ldw, void* workspace,
+pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, const void* f, pamm_index_type f_type,
+                                      const float* alpha, const void* dY, int64_t ldy, int64_t b, int64_t m,
+                                      pamm_dtype dt, int64_t k, float* Btilde, int64_t ldb, void* dW, int64_t ldw,
+                                      pamm_dtype dw_dt, pamm_layout layout, const void* sort_products, void* workspace,
                                       size_t ws_bytes, void* stream) {
-    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, false, workspace, ws_bytes);
+    pamm_status s = check_contract(f, f_type, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, false, sort_products, workspace, ws_bytes);
     if (s != PAMM_OK) return s;
-    const ContractWs w = contract_ws_layout(workspace, b, m, k);
+    const ContractWs w = contract_ws(workspace, b, m, k);
     float* Bt = Btilde ? Btilde : w.btilde;
     const int64_t ldbt = Btilde ? ldb : w.m_pad;
-    s = check_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dW, ldw);
+    const DwSpec dw = {dW, ldw, dw_dt, layout};
+    s = check_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dw);
     if (s != PAMM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
-    s = dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Bt, ldbt, w, st)
-                       : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Bt, ldbt, w, st);
+    const int32_t* pr = (const int32_t*)sort_products;
+    s = dt == PAMM_F32 ? launch_contract<float>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st)
+                       : launch_contract<__nv_bfloat16>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st);
     if (s != PAMM_OK) return s;
-    return do_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dW, ldw, st);
+    return do_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dw, st);
 }
 
 pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host, int64_t b, int64_t n, int64_t m,
@@ -509,10 +647,10 @@ pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host, int64_t 
         cudaMemcpy2DAsync(a.dY, a.ldy * es, dY_host, m * es, m * es, b, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return PAMM_ERR_CUDA;
     pamm_status s = pamm_compress_fused(a.X, a.ldx, b, n, dt, k, seed, nullptr, a.idx, a.C, a.ldc, a.invnorm, a.f,
-                                        a.alpha, nullptr, 0, stream);
+                                        PAMM_IDX_I32, a.alpha, a.products, sort_products_bytes(b, k), stream);
     if (s != PAMM_OK) return s;
-    s = pamm_contract_weight_grad(a.C, a.ldc, n, a.f, a.alpha, a.dY, a.ldy, b, m, dt, k, (float*)a.Bt, a.ldb,
-                                  (float*)a.dW, a.ldw, a.ws, a.ws_bytes, stream);
+    s = pamm_contract_weight_grad(a.C, a.ldc, n, a.f, PAMM_IDX_I32, a.alpha, a.dY, a.ldy, b, m, dt, k, (float*)a.Bt, a.ldb,
+                                  a.dW, a.ldw, PAMM_F32, PAMM_DW_NM, a.products, a.ws, a.ws_bytes, stream);
     if (s != PAMM_OK) return s;
     if (cudaMemcpy2DAsync(dW_host, m * 4, a.dW, a.ldw * 4, m * 4, n, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return PAMM_ERR_CUDA;
@@ -523,11 +661,46 @@ pamm_status pamm_qkv_step_host(const void* X_host, const void* dY_host, int64_t 
     return PAMM_OK;
 }
 
+// One small pinned host word and one private stream per device carry the status word
+// to the host without touching the caller's streams.
+namespace {
+struct StatusReader {
+    cudaStream_t stream = nullptr;
+    int* host_word = nullptr;
+    int* dev_word = nullptr;
+};
+StatusReader g_status_reader[64];
+std::mutex g_status_mutex;
+}  // namespace
+
 pamm_status pamm_last_device_status(void* stream) {
-    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PAMM_ERR_CUDA;
-    int word = 0, zero = 0;
-    if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int)) != cudaSuccess) return PAMM_ERR_CUDA;
-    if (word && cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)) != cudaSuccess) return PAMM_ERR_CUDA;
+    (void)stream;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return PAMM_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_status_mutex);
+    StatusReader& r = g_status_reader[dev];
+    if (!r.stream) {
+        void* sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess || !sym) return PAMM_ERR_CUDA;
+        if (cudaHostAlloc((void**)&r.host_word, sizeof(int), cudaHostAllocDefault) != cudaSuccess) return PAMM_ERR_CUDA;
+        if (cudaStreamCreateWithFlags(&r.stream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaFreeHost(r.host_word);
+            r.host_word = nullptr;
+            r.stream = nullptr;
+            return PAMM_ERR_CUDA;
+        }
+        r.dev_word = (int*)sym;
+    }
+    // a copy on the private stream: it waits for no kernel and blocks no stream of the caller
+    if (cudaMemcpyAsync(r.host_word, r.dev_word, sizeof(int), cudaMemcpyDeviceToHost, r.stream) != cudaSuccess ||
+        cudaStreamSynchronize(r.stream) != cudaSuccess)
+        return PAMM_ERR_CUDA;
+    const int word = *r.host_word;
+    if (word) {
+        if (cudaMemsetAsync(r.dev_word, 0, sizeof(int), r.stream) != cudaSuccess ||
+            cudaStreamSynchronize(r.stream) != cudaSuccess)
+            return PAMM_ERR_CUDA;
+    }
     if (word & DEV_TIMEOUT) return PAMM_ERR_TIMEOUT;
     if (word & DEV_BAD_INDEX) return PAMM_ERR_BAD_INDEX;
     return PAMM_OK;
@@ -566,14 +739,15 @@ extern "C" pamm_status pamm_contract_no_alloc(const int32_t* f, const float* alp
     // sizes first: the fixed array is the only scratch there is
     if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
     if (b < 1 || m < 1 || k < 1 || k > b || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
-    if (contract_ws_layout(nullptr, b, m, k).bytes > (size_t)PAMM_NO_ALLOC_SCRATCH_BYTES) return PAMM_ERR_WORKSPACE;
+    if (contract_ws(nullptr, b, m, k).bytes > (size_t)PAMM_NO_ALLOC_SCRATCH_BYTES) return PAMM_ERR_WORKSPACE;
     void* scratch = no_alloc_scratch_ptr();
     if (!scratch) return PAMM_ERR_CUDA;
-    pamm_status s = check_contract(f, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, scratch,
+    pamm_status s = check_contract(f, PAMM_IDX_I32, alpha, dY, ldy, b, m, dt, k, Btilde, ldb, true, nullptr, scratch,
                                    (size_t)PAMM_NO_ALLOC_SCRATCH_BYTES);
     if (s != PAMM_OK) return s;
-    const ContractWs w = contract_ws_layout(scratch, b, m, k);
+    const ContractWs w = contract_ws(scratch, b, m, k);
     cudaStream_t st = (cudaStream_t)stream;
-    return dt == PAMM_F32 ? launch_contract<float>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st)
-                          : launch_contract<__nv_bfloat16>(f, alpha, dY, ldy, b, m, k, Btilde, ldb, w, st);
+    return dt == PAMM_F32
+        ? launch_contract<float>(f, PAMM_IDX_I32, alpha, dY, ldy, b, m, k, Btilde, ldb, nullptr, w, st)
+        : launch_contract<__nv_bfloat16>(f, PAMM_IDX_I32, alpha, dY, ldy, b, m, k, Btilde, ldb, nullptr, w, st);
 }

@@ -11,10 +11,7 @@ from pathlib import Path
 
 import torch
 
-import os
-
-# PAMM_B200_LIB points the binding at another build of the same library (tuning builds).
-_LIB_PATH = Path(os.environ.get("PAMM_B200_LIB") or Path(__file__).resolve().parent / "libpamm_b200.so")
+_LIB_PATH = Path(__file__).resolve().parent / "libpamm_b200.so"
 if not _LIB_PATH.exists():
     raise ImportError(
         f"{_LIB_PATH} is missing: build it with `python -m paper_2506_02939_b200.build` "
@@ -23,6 +20,8 @@ _lib = ctypes.CDLL(str(_LIB_PATH))
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_INDEX = range(7)
 F32, BF16 = 0, 1
+DW_NM, DW_MN = 0, 1                      # layout of the weight gradient: n x m (the paper's), or m x n (out x in)
+IDX_I32, IDX_U16, IDX_U8 = 0, 1, 2       # storage type of the assignment f
 WS_COMPRESS, WS_CONTRACT, WS_STEP_HOST = 0, 1, 2
 
 _i64, _vp, _ci, _u64, _sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_uint64, ctypes.c_size_t
@@ -30,17 +29,21 @@ _i64, _vp, _ci, _u64, _sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctype
 _SIGNATURES = {
     "pamm_status_string": ([_ci], ctypes.c_char_p),
     "pamm_version": ([], _ci),
+    "pamm_last_error_detail": ([], ctypes.c_char_p),
     "pamm_workspace_bytes": ([_ci, _i64, _i64, _i64, _i64, _ci], _sz),
+    "pamm_saved_bytes": ([_i64, _i64, _i64, _ci, _ci, _vp], _ci),
     "pamm_draw_indices_host": ([_i64, _i64, _u64, _vp], _ci),
     "pamm_select_generators": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp], _ci),
-    "pamm_compress": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
-    "pamm_compress_fused": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
-    "pamm_contract": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
-    "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
-    "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
-    "pamm_weight_grad_beta": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _i64, _vp], _ci),
-    "pamm_weight_grad_accumulate": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _vp], _ci),
-    "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64, _vp, _sz, _vp], _ci),
+    "pamm_compress": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _vp, _ci, _vp, _vp, _sz, _vp], _ci),
+    "pamm_compress_fused": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _ci, _vp, _vp, _sz, _vp], _ci),
+    "pamm_compress_projections": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _ci, _vp, _i64, _vp, _sz, _vp], _ci),
+    "pamm_contract": ([_vp, _ci, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _vp, _sz, _vp], _ci),
+    "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _ci, _ci, _vp], _ci),
+    "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _ci, _vp, _vp, _vp, _sz, _vp], _ci),
+    "pamm_weight_grad_beta": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _i64, _ci, _ci, _vp], _ci),
+    "pamm_weight_grad_accumulate": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _ci, _vp], _ci),
+    "pamm_contract_weight_grad": ([_vp, _i64, _i64, _vp, _ci, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _i64,
+                                   _ci, _ci, _vp, _vp, _sz, _vp], _ci),
     "pamm_qkv_step_host": ([_vp, _vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _vp, _sz, _vp], _ci),
     "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
     "pamm_last_device_status": ([_vp], _ci),
@@ -58,7 +61,8 @@ EXPORTED = tuple(_SIGNATURES)
 class PammError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {status_string(code)} (status {code})")
+        detail = _lib.pamm_last_error_detail().decode() if code == ERR_CUDA else ""
+        super().__init__(f"{where}: {status_string(code)} (status {code})" + (f": {detail}" if detail else ""))
 
 
 def status_string(code: int) -> str:
@@ -131,72 +135,123 @@ def select_generators(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=Non
     return idx_out, C, c_invnorm
 
 
-def compress(X, C, c_invnorm, f=None, alpha=None, workspace=None, stream=None):
+_F_TYPES = {torch.int32: IDX_I32, torch.uint16: IDX_U16, torch.int16: IDX_U16, torch.uint8: IDX_U8}
+
+
+def _ft(f: torch.Tensor) -> int:
+    """Storage type of an assignment vector (narrow entries are unsigned whatever torch calls them)."""
+    try:
+        return _F_TYPES[f.dtype]
+    except KeyError:
+        raise TypeError(f"f is int32, uint16 (or int16 storage) or uint8, got {f.dtype}") from None
+
+
+def _new_f(shape, f_dtype, device):
+    return torch.empty(shape, dtype=torch.int32 if f_dtype is None else f_dtype, device=device)
+
+
+def _bytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def compress(X, C, c_invnorm, f=None, alpha=None, sort_products=None, f_dtype=None, stream=None):
+    """``sort_products``: optional uint8 tensor of ``workspace_bytes(WS_COMPRESS, ...)`` bytes that receives the
+    per-block counts of f for the backward pass."""
     b, n = X.shape
     k = C.shape[0]
-    f = torch.empty(b, dtype=torch.int32, device=X.device) if f is None else f
+    f = _new_f(b, f_dtype, X.device) if f is None else f
     alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
-    ws_bytes = 0 if workspace is None else workspace.numel()
-    _check(_lib.pamm_compress(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), _ptr(f),
-                              _ptr(alpha), _ptr(workspace), ws_bytes, _stream(stream)), "pamm_compress")
+    _check(_lib.pamm_compress(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), _ptr(f), _ft(f),
+                              _ptr(alpha), _ptr(sort_products), _bytes(sort_products), _stream(stream)), "pamm_compress")
     return f, alpha
 
 
-def compress_eps(X, C, c_invnorm, eps: float, f=None, alpha=None, dropped=None, stream=None):
+def compress_projections(X, C, c_invnorm, sets: int, f=None, alpha=None, sort_products=None, f_dtype=None, stream=None):
+    """One compression per projection in one pass over X: ``C`` holds ``sets * k`` generator rows and ``c_invnorm``
+    ``sets * 2k`` norms (one ``select_generators`` call per set); returns f and alpha of shape (sets, b)."""
+    b, n = X.shape
+    k = C.shape[0] // sets
+    f = _new_f((sets, b), f_dtype, X.device) if f is None else f
+    alpha = torch.empty((sets, b), dtype=torch.float32, device=X.device) if alpha is None else alpha
+    _check(_lib.pamm_compress_projections(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, sets, _ptr(c_invnorm), _ptr(f),
+                                          _ft(f), _ptr(alpha), f.stride(0), _ptr(sort_products), _bytes(sort_products),
+                                          _stream(stream)), "pamm_compress_projections")
+    return f, alpha
+
+
+def compress_eps(X, C, c_invnorm, eps: float, f=None, alpha=None, dropped=None, sort_products=None, f_dtype=None,
+                 stream=None):
     """compress with the neighbourhood condition (Eq. 2): rows farther than eps ||X_i|| from their representative
     get alpha = 0; ``dropped`` (device int32[1]) receives their number."""
     b, n = X.shape
     k = C.shape[0]
-    f = torch.empty(b, dtype=torch.int32, device=X.device) if f is None else f
+    f = _new_f(b, f_dtype, X.device) if f is None else f
     alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
     dropped = torch.empty(1, dtype=torch.int32, device=X.device) if dropped is None else dropped
     _check(_lib.pamm_compress_eps(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), float(eps), _ptr(f),
-                                  _ptr(alpha), _ptr(dropped), None, 0, _stream(stream)), "pamm_compress_eps")
+                                  _ft(f), _ptr(alpha), _ptr(dropped), _ptr(sort_products), _bytes(sort_products),
+                                  _stream(stream)), "pamm_compress_eps")
     return f, alpha, dropped
 
 
-def weight_grad_beta(C, Btilde, b: int, dropped, dW=None, stream=None):
-    """dW = beta C^T B~ with beta = b / (b - eta), eta read from ``dropped`` on the device (Eq. 4-5)."""
+def _new_dW(n: int, m: int, dw_dtype, layout: int, device):
+    rows, cols = (m, n) if layout == DW_MN else (n, m)
+    return alloc_matrix(rows, cols, torch.float32 if dw_dtype is None else dw_dtype, device)
+
+
+def weight_grad(C, Btilde, dW=None, dw_dtype=None, layout: int = DW_NM, stream=None):
+    """dW = C^T B~: n x m (``DW_NM``) or its transpose m x n (``DW_MN``), fp32 or bf16."""
     k, n = C.shape
     m = Btilde.shape[1]
-    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
-    _check(_lib.pamm_weight_grad_beta(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, b, _ptr(dropped),
-                                      _ptr(dW), _ld(dW), _stream(stream)), "pamm_weight_grad_beta")
+    dW = _new_dW(n, m, dw_dtype, layout, C.device) if dW is None else dW
+    _check(_lib.pamm_weight_grad(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW), _dt(dW),
+                                 layout, _stream(stream)), "pamm_weight_grad")
     return dW
 
 
-def weight_grad_accumulate(C, Btilde, dW, stream=None):
-    """dW += C^T B~ (gradient accumulation over micro-batches)."""
+def weight_grad_beta(C, Btilde, b: int, dropped, dW=None, dw_dtype=None, layout: int = DW_NM, stream=None):
+    """dW = beta C^T B~ with beta = b / (b - eta), eta read from ``dropped`` on the device (Eq. 4-5)."""
     k, n = C.shape
     m = Btilde.shape[1]
+    dW = _new_dW(n, m, dw_dtype, layout, C.device) if dW is None else dW
+    _check(_lib.pamm_weight_grad_beta(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, b, _ptr(dropped),
+                                      _ptr(dW), _ld(dW), _dt(dW), layout, _stream(stream)), "pamm_weight_grad_beta")
+    return dW
+
+
+def weight_grad_accumulate(C, Btilde, dW, layout: int = DW_NM, stream=None):
+    """dW += C^T B~ (gradient accumulation over micro-batches); dW is fp32."""
+    k, n = C.shape
+    m = Btilde.shape[1]
+    if dW.dtype != torch.float32:
+        raise TypeError("gradients are accumulated in float32")
     _check(_lib.pamm_weight_grad_accumulate(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW),
-                                            _stream(stream)), "pamm_weight_grad_accumulate")
+                                            layout, _stream(stream)), "pamm_weight_grad_accumulate")
     return dW
 
 
 def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, f=None, alpha=None,
-                   workspace=None, stream=None):
+                   sort_products=None, f_dtype=None, stream=None):
     b, n = X.shape
     dev = X.device
     idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
     C = alloc_matrix(k, n, X.dtype, dev) if C is None else C
     c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
-    f = torch.empty(b, dtype=torch.int32, device=dev) if f is None else f
+    f = _new_f(b, f_dtype, dev) if f is None else f
     alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
-    ws_bytes = 0 if workspace is None else workspace.numel()
     _check(_lib.pamm_compress_fused(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out), _ptr(C),
-                                    _ld(C), _ptr(c_invnorm), _ptr(f), _ptr(alpha), _ptr(workspace), ws_bytes,
-                                    _stream(stream)), "pamm_compress_fused")
+                                    _ld(C), _ptr(c_invnorm), _ptr(f), _ft(f), _ptr(alpha), _ptr(sort_products),
+                                    _bytes(sort_products), _stream(stream)), "pamm_compress_fused")
     return idx_out, C, c_invnorm, f, alpha
 
 
-def contract(f, alpha, dY, k: int, Btilde=None, workspace=None, stream=None):
+def contract(f, alpha, dY, k: int, Btilde=None, sort_products=None, workspace=None, stream=None):
     b, m = dY.shape
     Btilde = alloc_matrix(k, m, torch.float32, dY.device) if Btilde is None else Btilde
     if workspace is None:
         workspace = alloc_workspace(WS_CONTRACT, b, 1, m, k, _dt(dY), dY.device)
-    _check(_lib.pamm_contract(_ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde), _ld(Btilde),
-                              _ptr(workspace), workspace.numel(), _stream(stream)), "pamm_contract")
+    _check(_lib.pamm_contract(_ptr(f), _ft(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY), k, _ptr(Btilde), _ld(Btilde),
+                              _ptr(sort_products), _ptr(workspace), workspace.numel(), _stream(stream)), "pamm_contract")
     return Btilde
 
 
@@ -216,24 +271,16 @@ def contract_no_alloc(f, alpha, dY, k: int, Btilde, stream=None):
     return Btilde
 
 
-def weight_grad(C, Btilde, dW=None, stream=None):
-    k, n = C.shape
-    m = Btilde.shape[1]
-    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
-    _check(_lib.pamm_weight_grad(_ptr(C), _ld(C), k, n, _dt(C), _ptr(Btilde), _ld(Btilde), m, _ptr(dW), _ld(dW),
-                                 _stream(stream)), "pamm_weight_grad")
-    return dW
-
-
-def contract_weight_grad(C, f, alpha, dY, Btilde=None, dW=None, workspace=None, stream=None):
+def contract_weight_grad(C, f, alpha, dY, Btilde=None, dW=None, dw_dtype=None, layout: int = DW_NM, sort_products=None,
+                         workspace=None, stream=None):
     k, n = C.shape
     b, m = dY.shape
-    dW = alloc_matrix(n, m, torch.float32, C.device) if dW is None else dW
+    dW = _new_dW(n, m, dw_dtype, layout, C.device) if dW is None else dW
     if workspace is None:
         workspace = alloc_workspace(WS_CONTRACT, b, n, m, k, _dt(dY), dY.device)
-    _check(_lib.pamm_contract_weight_grad(_ptr(C), _ld(C), n, _ptr(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY),
-                                          k, _ptr(Btilde), 0 if Btilde is None else _ld(Btilde), _ptr(dW), _ld(dW),
-                                          _ptr(workspace), workspace.numel(), _stream(stream)),
+    _check(_lib.pamm_contract_weight_grad(_ptr(C), _ld(C), n, _ptr(f), _ft(f), _ptr(alpha), _ptr(dY), _ld(dY), b, m, _dt(dY),
+                                          k, _ptr(Btilde), 0 if Btilde is None else _ld(Btilde), _ptr(dW), _ld(dW), _dt(dW),
+                                          layout, _ptr(sort_products), _ptr(workspace), workspace.numel(), _stream(stream)),
            "pamm_contract_weight_grad")
     return dW
 
@@ -255,8 +302,13 @@ def selftest_bounded_wait(stream=None) -> None:
     _check(_lib.pamm_selftest_bounded_wait(_stream(stream)), "pamm_selftest_bounded_wait")
 
 
-def last_device_status(stream=None) -> int:
-    return int(_lib.pamm_last_device_status(_stream(stream)))
+def last_device_status(stream=None, synchronize: bool = True) -> int:
+    """The device's status word, read and cleared.  The library call itself waits for nothing; by default the
+    given (or current) stream is synchronised first, so that the answer covers the work enqueued so far."""
+    s = torch.cuda.current_stream() if stream is None else stream
+    if synchronize:
+        s.synchronize()
+    return int(_lib.pamm_last_device_status(ctypes.c_void_p(s.cuda_stream)))
 
 
 PROF_COMPRESS, PROF_CONTRACT, PROF_WEIGHT_GRAD = 0, 1, 2
@@ -273,9 +325,8 @@ def set_profile_events(kind: int, start=None, stop=None) -> None:
     _check(_lib.pamm_set_profile_events(kind, a, b), "pamm_set_profile_events")
 
 
-def saved_bytes(b: int, n: int, k: int, dtype: int) -> dict:
-    """Bytes kept for the backward pass: X itself versus (C, f int32, alpha fp32)."""
-    e = 2 if dtype == BF16 else 4
-    full = b * n * e
-    kept = k * n * e + 8 * b
-    return dict(full=full, pamm=kept, ratio=full / kept, scalars_full=b * n, scalars_pamm=k * n + 2 * b)
+def saved_bytes(b: int, n: int, k: int, dtype: int, f_type: int = IDX_I32) -> dict:
+    """Bytes kept for the backward pass: X itself versus (C, f, alpha); and the paper's scalar counts."""
+    out = (ctypes.c_int64 * 4)()
+    _check(_lib.pamm_saved_bytes(b, n, k, dtype, f_type, ctypes.cast(out, ctypes.c_void_p)), "pamm_saved_bytes")
+    return dict(full=int(out[0]), pamm=int(out[1]), ratio=out[0] / out[1], scalars_full=int(out[2]), scalars_pamm=int(out[3]))

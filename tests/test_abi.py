@@ -34,6 +34,18 @@ def test_version_and_status_strings():
     assert len(seen) == 7 and "ok" in seen
 
 
+def test_saved_bytes_follow_the_papers_count():
+    # appendix "Complexity Analysis": k n + 2 b scalars instead of b n
+    s = pamm.saved_bytes(65536, 2048, 128, pamm.BF16)
+    assert s["scalars_full"] == 65536 * 2048 and s["scalars_pamm"] == 128 * 2048 + 2 * 65536
+    assert s["full"] == 65536 * 2048 * 2 and s["pamm"] == 128 * 2048 * 2 + 8 * 65536
+    assert abs(s["ratio"] - 256.0) < 1e-9
+    narrow = pamm.saved_bytes(65536, 2048, 128, pamm.BF16, pamm.IDX_U8)
+    assert narrow["pamm"] == 128 * 2048 * 2 + 5 * 65536
+    with pytest.raises(pamm.PammError):
+        pamm.saved_bytes(65536, 2048, 300, pamm.BF16, pamm.IDX_U8)      # 300 generators do not fit a byte
+
+
 def test_workspace_sizes():
     w = pamm.workspace_bytes(pamm.WS_CONTRACT, 65536, 2048, 6144, 128, pamm.BF16)
     assert w % 256 == 0 and 0 < w < 64 << 20
@@ -41,6 +53,9 @@ def test_workspace_sizes():
     assert pamm.workspace_bytes(pamm.WS_CONTRACT, 65536, 2048, 6144, 256, pamm.BF16) > w
     assert pamm.workspace_bytes(pamm.WS_CONTRACT, 65536, 2048, 12288, 128, pamm.BF16) > w
     assert pamm.workspace_bytes(pamm.WS_STEP_HOST, 2048, 512, 1536, 4, pamm.F32) > 2048 * (512 + 1536) * 4
+    # the sort products: one count per generator and block of rows, at most one block per SM
+    p = pamm.workspace_bytes(pamm.WS_COMPRESS, 65536, 2048, 6144, 128, pamm.BF16)
+    assert p % 256 == 0 and 128 * 4 <= p <= 256 * 128 * 4
     with pytest.raises(pamm.PammError):
         pamm.workspace_bytes(pamm.WS_CONTRACT, 16, 8, 8, 17, pamm.F32)     # k > b
     with pytest.raises(pamm.PammError):
@@ -61,22 +76,36 @@ def test_argument_errors_are_synchronous_and_launch_nothing():
     # k > b, k < 1
     assert i.pamm_select_generators(fake, 8, 16, 8, pamm.F32, 17, 0, null, fake, fake, 8, fake, null) == pamm.ERR_INVALID_ARG
     assert i.pamm_select_generators(fake, 8, 16, 8, pamm.F32, 0, 0, null, fake, fake, 8, fake, null) == pamm.ERR_INVALID_ARG
+    I32, U8 = pamm.IDX_I32, pamm.IDX_U8
     # ld < n and ld not a multiple of 16 bytes
-    assert i.pamm_compress(fake, 4, 16, 8, pamm.F32, fake, 8, 2, fake, fake, fake, null, 0, null) == pamm.ERR_INVALID_ARG
-    assert i.pamm_compress(fake, 9, 16, 8, pamm.F32, fake, 8, 2, fake, fake, fake, null, 0, null) == pamm.ERR_INVALID_ARG
-    assert i.pamm_compress(fake, 12, 16, 8, pamm.BF16, fake, 8, 2, fake, fake, fake, null, 0, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_compress(fake, 4, 16, 8, pamm.F32, fake, 8, 2, fake, fake, I32, fake, null, 0, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_compress(fake, 9, 16, 8, pamm.F32, fake, 8, 2, fake, fake, I32, fake, null, 0, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_compress(fake, 12, 16, 8, pamm.BF16, fake, 8, 2, fake, fake, I32, fake, null, 0, null) == pamm.ERR_INVALID_ARG
     # misaligned base pointer
-    assert i.pamm_compress(odd, 8, 16, 8, pamm.F32, fake, 8, 2, fake, fake, fake, null, 0, null) == pamm.ERR_INVALID_ARG
-    # unknown dtype
-    assert i.pamm_compress(fake, 8, 16, 8, 7, fake, 8, 2, fake, fake, fake, null, 0, null) == pamm.ERR_UNSUPPORTED
+    assert i.pamm_compress(odd, 8, 16, 8, pamm.F32, fake, 8, 2, fake, fake, I32, fake, null, 0, null) == pamm.ERR_INVALID_ARG
+    # unknown dtype, unknown storage type of f
+    assert i.pamm_compress(fake, 8, 16, 8, 7, fake, 8, 2, fake, fake, I32, fake, null, 0, null) == pamm.ERR_UNSUPPORTED
+    assert i.pamm_compress(fake, 8, 16, 8, pamm.F32, fake, 8, 2, fake, fake, 9, fake, null, 0, null) == pamm.ERR_UNSUPPORTED
+    # more generators than the storage type of f can name
+    assert i.pamm_compress(fake, 8, 1000, 8, pamm.F32, fake, 8, 257, fake, fake, U8, fake, null, 0, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_contract(fake, U8, fake, fake, 8, 1000, 8, pamm.F32, 257, fake, 8, null, fake, 1 << 30, null) == pamm.ERR_INVALID_ARG
+    # a buffer for the sort products that is too small or misaligned
+    assert i.pamm_compress(fake, 8, 16, 8, pamm.F32, fake, 8, 2, fake, fake, I32, fake, fake, 8, null) == pamm.ERR_WORKSPACE
+    assert i.pamm_compress(fake, 8, 16, 8, pamm.F32, fake, 8, 2, fake, fake, I32, fake, odd, 1 << 20, null) == pamm.ERR_WORKSPACE
     # contract: missing / small / misaligned workspace
-    assert i.pamm_contract(fake, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, null, 0, null) == pamm.ERR_WORKSPACE
-    assert i.pamm_contract(fake, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, fake, 16, null) == pamm.ERR_WORKSPACE
-    assert i.pamm_contract(fake, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, odd, 1 << 20, null) == pamm.ERR_WORKSPACE
-    assert i.pamm_contract(fake, fake, fake, 8, 16, 8, pamm.F32, 2, null, 8, fake, 1 << 20, null) == pamm.ERR_INVALID_ARG
-    # weight grad
-    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 8, 8, null, 8, null) == pamm.ERR_INVALID_ARG
-    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 6, 8, fake, 8, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_contract(fake, I32, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, null, null, 0, null) == pamm.ERR_WORKSPACE
+    assert i.pamm_contract(fake, I32, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, null, fake, 16, null) == pamm.ERR_WORKSPACE
+    assert i.pamm_contract(fake, I32, fake, fake, 8, 16, 8, pamm.F32, 2, fake, 8, null, odd, 1 << 20, null) == pamm.ERR_WORKSPACE
+    assert i.pamm_contract(fake, I32, fake, fake, 8, 16, 8, pamm.F32, 2, null, 8, null, fake, 1 << 20, null) == pamm.ERR_INVALID_ARG
+    # weight grad: NULL output, bad leading dimension of B~, unknown output type / layout, bf16 accumulate is not offered
+    NM, MN = pamm.DW_NM, pamm.DW_MN
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 8, 8, null, 8, pamm.F32, NM, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 6, 8, fake, 8, pamm.F32, NM, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 8, 8, fake, 8, 5, NM, null) == pamm.ERR_UNSUPPORTED
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 8, 8, fake, 8, pamm.F32, 3, null) == pamm.ERR_UNSUPPORTED
+    # the leading dimension of dW counts the columns of the chosen layout: n = 8, m = 24
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 24, 24, fake, 8, pamm.F32, NM, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_weight_grad(fake, 8, 2, 8, pamm.F32, fake, 24, 24, fake, 12, pamm.BF16, MN, null) == pamm.ERR_INVALID_ARG
     # host step: arena too small
     assert i.pamm_qkv_step_host(fake, fake, 16, 8, 8, pamm.F32, 2, 0, fake, null, null, fake, 64, null) == pamm.ERR_WORKSPACE
     # limits

@@ -21,7 +21,8 @@ def test_forward_and_input_gradient_are_exact_weight_gradient_is_pamm():
     Z = PammLinearFunction.apply(X, W, 32, 7)
     assert torch.equal(Z, X.detach() @ W.detach())
     kept = Z.grad_fn.saved_tensors
-    assert len(kept) == 4 and all(t.numel() < X.numel() // 4 or t is W for t in kept)   # X itself is not kept
+    assert len(kept) == 5 and all(t.numel() * t.element_size() < X.numel() * 2 // 4 or t is W for t in kept)   # X itself is not kept
+    assert kept[1].dtype == torch.uint8                                          # 32 generators: a byte per row names one
     dZ = parity.to_device(dZn).reshape(4, 256, 384)
     Z.backward(dZ)
     assert torch.equal(X.grad, dZ @ W.detach().t())

@@ -80,6 +80,13 @@ def test_neighbourhood_parity(b, n, m, k, dtype, eps):
     print(dtype, b, n, k, eps, {q: r[q] for q in ("kept", "eta", "window", "disagree")})
 
 
+def test_largest_generator_count_with_the_row_norm_warps():
+    # k = 4096 leaves the least shared memory for the pipeline: the stage count gives way, not the launch
+    X, dY = synth.random_case(4500, 128, 72, "bf16", seed=91, centres=300, noise=0.25, dy_scale=1e-3)
+    r = run_eps(X, dY, 4096, 0.2)
+    assert r["eta"] > 0
+
+
 def test_both_branches_are_exercised():
     X, dY = synth.random_case(3000, 200, 264, "bf16", seed=77, centres=12, noise=0.25, dy_scale=1e-3)
     r = run_eps(X, dY, 40, 0.3)

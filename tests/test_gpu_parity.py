@@ -46,15 +46,15 @@ def test_small_cases(b, n, m, k, dtype, fused):
 def test_many_rows_ragged_everywhere():
     # more rows than 148 x 1024 (several sort blocks per SM, ranges of ~1350 rows per CTA), nothing a multiple of a tile
     X, dY = synth.random_case(200003, 264, 520, "bf16", seed=51, centres=40, dy_scale=1e-3)
-    rep = parity.run_and_compare(X, dY, 96, seed=52, full_dW=False)
+    rep = parity.run_and_compare(X, dY, 96, seed=52, products=True)
     assert rep.unexplained == 0
 
 
 def test_largest_generator_count_of_the_tensor_core_path():
     # k = 4096: sixteen chunks of 256 generators with a running argmax per row; k = 4097 takes the CUDA-core path
     X, dY = synth.random_case(4500, 128, 72, "bf16", seed=53, centres=300, dy_scale=1e-3)
-    parity.run_and_compare(X, dY, 4096, seed=54, full_dW=False)
-    parity.run_and_compare(X[:4200], dY[:4200], 4097, seed=55, full_dW=False)
+    parity.run_and_compare(X, dY, 4096, seed=54, products=True)
+    parity.run_and_compare(X[:4200], dY[:4200], 4097, seed=55)
 
 
 def test_ragged_columns_with_padded_leading_dimension():
@@ -225,16 +225,16 @@ def test_host_buffer_step_matches_device_path():
 def test_workload_full_size(name):
     inp = synth.make_inputs(name)
     w = inp.workload
-    rep = parity.run_and_compare(inp.X, inp.dY, w.ks[0], seed=w.index_seed)
-    print(name, rep.err, "mismatch", rep.mismatches, "near-tie", rep.near_tie, "rounding", rep.explained_by_rounding)
+    rep = parity.run_and_compare(inp.X, inp.dY, w.ks[0], seed=w.index_seed, products=True)
+    parity.record(f"{name} k={w.ks[0]}", rep)
 
 
 def test_workload_c3_ratio_sweep():
     inp = synth.make_inputs("c3")
     w = inp.workload
     for k in w.ks:
-        rep = parity.run_and_compare(inp.X, inp.dY, k, seed=w.index_seed)
-        print("c3", k, rep.err, "mismatch", rep.mismatches, "near-tie", rep.near_tie, "rounding", rep.explained_by_rounding)
+        rep = parity.run_and_compare(inp.X, inp.dY, k, seed=w.index_seed, products=True)
+        parity.record(f"c3 k={k}", rep)
 
 
 def test_layer_stack_keeps_only_the_compressed_state():
@@ -266,20 +266,165 @@ def test_layer_stack_keeps_only_the_compressed_state():
         assert parity.rel_fro(dW[rr, cc], ref) <= 1e-2
 
 
+@pytest.mark.parametrize("layout", [pamm.DW_NM, pamm.DW_MN])
 @pytest.mark.parametrize("k,n,m,dtype", [(24, 136, 264, "bf16"), (200, 72, 136, "bf16"), (5, 40, 52, "f32")])
-def test_weight_grad_accumulate_adds_to_dW(k, n, m, dtype):
-    # the three product kernels (persistent tcgen05, one-tile tcgen05, CUDA cores): dW += C^T B~, twice
+def test_weight_grad_accumulate_adds_to_dW(k, n, m, dtype, layout):
+    # the three product kernels (persistent tcgen05, chunked tcgen05, CUDA cores): dW += C^T B~, twice, either layout
     Cb, _ = synth.random_case(k, n, 8, dtype, seed=21)
     Bt = torch.from_numpy(np.random.default_rng(22).standard_normal((k, m)).astype(np.float32)).cuda()
     C = parity.to_device(Cb)
-    base = torch.from_numpy(np.random.default_rng(23).standard_normal((n, m)).astype(np.float32)).cuda()
-    once = pamm.weight_grad(C, Bt)
+    shape = (n, m) if layout == pamm.DW_NM else (m, n)
+    base = torch.from_numpy(np.random.default_rng(23).standard_normal(shape).astype(np.float32)).cuda()
+    once = pamm.weight_grad(C, Bt, layout=layout)
+    assert once.shape == shape
     dW = base.clone()
-    pamm.weight_grad_accumulate(C, Bt, dW)
+    pamm.weight_grad_accumulate(C, Bt, dW, layout=layout)
     assert torch.allclose(dW, base + once, rtol=1e-6, atol=1e-6)
-    pamm.weight_grad_accumulate(C, Bt, dW)
+    pamm.weight_grad_accumulate(C, Bt, dW, layout=layout)
     assert torch.allclose(dW, base + 2 * once, rtol=1e-6, atol=1e-5)
     assert pamm.last_device_status() == pamm.OK
+
+
+# ---- storage options of the outputs: dW in fp32 / bf16, n x m / m x n; f in 32 / 16 / 8 bits ----
+
+@pytest.mark.parametrize("layout", [pamm.DW_NM, pamm.DW_MN])
+@pytest.mark.parametrize("dw_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("b,n,m,k,dtype", [
+    (1500, 264, 392, 48, "bf16"),      # persistent tcgen05 product (k <= 128), ragged tiles in both directions
+    (1200, 136, 200, 200, "bf16"),     # chunked tcgen05 product (k > 128)
+    (900, 72, 100, 5, "f32"),          # CUDA-core product
+    (700, 40, 56, 6, "bf16"),          # bf16 generators with k < 8: CUDA-core product
+])
+def test_weight_gradient_types_and_layouts(b, n, m, k, dtype, dw_dtype, layout):
+    X, dY = synth.random_case(b, n, m, dtype, seed=31 + k, centres=max(2, k // 2), dy_scale=1e-3)
+    rep = parity.run_and_compare(X, dY, k, seed=3 + k, dw_dtype=dw_dtype, layout=layout)
+    assert rep.unexplained == 0
+
+
+def test_fp32_weight_gradient_in_the_papers_layout_is_unchanged_by_the_options():
+    # the transposed layout holds the same numbers; the bf16 one their nearest-even roundings
+    X, dY = synth.random_case(2000, 264, 392, "bf16", seed=41, centres=12, dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    for k in (48, 200):
+        idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, 5)
+        Bt = pamm.contract(f, alpha, dYd, k)
+        ref = pamm.weight_grad(C, Bt)
+        assert torch.equal(pamm.weight_grad(C, Bt, layout=pamm.DW_MN).t(), ref)
+        assert torch.equal(pamm.weight_grad(C, Bt, dw_dtype=torch.bfloat16), ref.to(torch.bfloat16))
+        assert torch.equal(pamm.weight_grad(C, Bt, dw_dtype=torch.bfloat16, layout=pamm.DW_MN).t(), ref.to(torch.bfloat16))
+    assert pamm.last_device_status() == pamm.OK
+
+
+@pytest.mark.parametrize("f_dtype,b,n,m,k,dtype", [
+    (torch.uint8, 3000, 136, 264, 200, "bf16"),
+    (torch.uint8, 1000, 72, 40, 256, "bf16"),         # the largest k a byte can name
+    (torch.int16, 2500, 200, 136, 700, "bf16"),       # unsigned 16-bit entries (torch's int16 as storage)
+    (torch.uint8, 800, 64, 48, 3, "f32"),             # CUDA-core compress
+])
+def test_narrow_assignment_storage(f_dtype, b, n, m, k, dtype):
+    X, dY = synth.random_case(b, n, m, dtype, seed=17 + k, centres=max(2, k // 2), dy_scale=1e-3)
+    for fused in (True, False):
+        rep = parity.run_and_compare(X, dY, k, seed=2 + k, f_dtype=f_dtype, fused=fused, products=fused)
+        assert rep.unexplained == 0
+    # and the same bits as the 32-bit path
+    Xd = parity.to_device(X)
+    _, C, invn, f32, a32 = pamm.compress_fused(Xd, k, 9)
+    _, _, _, fn, an = pamm.compress_fused(Xd, k, 9, f_dtype=f_dtype)
+    wide = fn.to(torch.int32) & (0xFFFF if f_dtype == torch.int16 else 0xFF)
+    assert torch.equal(wide, f32) and torch.equal(an, a32)
+    with pytest.raises(pamm.PammError):
+        pamm.compress_fused(Xd, 257, 9, f_dtype=torch.uint8)
+
+
+# ---- the counts of f that the forward pass leaves for the backward pass ----
+
+@pytest.mark.parametrize("b,n,m,k,dtype", [(5000, 136, 264, 40, "bf16"), (3000, 64, 72, 900, "bf16"), (2048, 72, 96, 4, "f32")])
+def test_sort_products_of_the_forward_pass(b, n, m, k, dtype):
+    # tensor-core compress, the three-launch sort (many generators), CUDA-core compress
+    X, dY = synth.random_case(b, n, m, dtype, seed=61, centres=max(2, k // 3), dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    code = pamm.BF16 if dtype == "bf16" else pamm.F32
+    sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, code)
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, 4, sort_products=sp)
+    # the products are histograms of f per block of rows (equal blocks, at most one per SM, a multiple of 64 rows):
+    # their column sums are the histogram of the whole f
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rows_per_block = max(64, (-(-b // sms) + 63) // 64 * 64)
+    nblk = -(-b // rows_per_block)
+    counts = sp[: nblk * k * 4].view(torch.int32).view(nblk, k).to(torch.int64)
+    assert torch.equal(counts.sum(dim=0), torch.bincount(f.to(torch.int64), minlength=k))
+    assert torch.equal(counts[0], torch.bincount(f[:rows_per_block].to(torch.int64), minlength=k))
+    launches0 = pamm.launch_count()
+    with_products = pamm.contract(f, alpha, dYd, k, sort_products=sp)
+    n_with = pamm.launch_count() - launches0
+    launches0 = pamm.launch_count()
+    without = pamm.contract(f, alpha, dYd, k)
+    n_without = pamm.launch_count() - launches0
+    assert n_with == n_without - 1                                   # the counting launch is gone
+    assert torch.equal(with_products, without)
+    assert pamm.last_device_status() == pamm.OK
+
+
+def test_sort_products_of_another_assignment_are_reported_not_trusted():
+    X, dY = synth.random_case(4000, 72, 136, "bf16", seed=62, centres=9, dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    k = 24
+    sp = pamm.alloc_workspace(pamm.WS_COMPRESS, 4000, 72, 136, k, pamm.BF16)
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, 4, sort_products=sp)
+    sp.view(torch.int32)[: 6 * k] += 1000                            # counts that do not belong to f any more
+    Bt = pamm.contract(f, alpha, dYd, k, sort_products=sp)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX           # noticed on the device, nothing faulted
+    assert pamm.last_device_status() == pamm.OK
+    good = pamm.contract(f, alpha, dYd, k)                           # and the library carries on
+    ref = orc.contract(f.cpu().numpy(), alpha.cpu().numpy().astype(np.float64), dY, k)
+    assert parity.rel_fro(good.cpu().numpy(), ref) <= 1e-5
+
+
+# ---- one compression per projection, in one pass over X (Section 4) ----
+
+@pytest.mark.parametrize("b,n,k,dtype,sets", [(3000, 264, 40, "bf16", 3), (2000, 136, 300, "bf16", 3), (1500, 72, 5, "f32", 3),
+                                              (1000, 64, 100, "bf16", 2)])
+def test_one_compression_per_projection(b, n, k, dtype, sets):
+    ms = [136, 72, 40][:sets]
+    m = sum(ms)
+    X, dY = synth.random_case(b, n, m, dtype, seed=71 + k, centres=max(3, k // 2), dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    tdt = Xd.dtype
+    C = pamm.alloc_matrix(sets * k, n, tdt)
+    invn = torch.empty(sets * 2 * k, dtype=torch.float32, device="cuda")
+    idx = torch.empty(sets * k, dtype=torch.int32, device="cuda")
+    for s in range(sets):                                            # an index seed per projection
+        pamm.select_generators(Xd, k, seed=100 + s, idx_out=idx[s * k:(s + 1) * k], C=C[s * k:(s + 1) * k],
+                               c_invnorm=invn[s * 2 * k:(s + 1) * 2 * k])
+    f, alpha = pamm.compress_projections(Xd, C, invn, sets)
+    assert f.shape == (sets, b) and alpha.shape == (sets, b)
+    dW = pamm.alloc_matrix(n, m, torch.float32)
+    col = 0
+    for s in range(sets):
+        # every set's result is what a compression of its own gives, bit for bit
+        f1, a1 = pamm.compress(Xd, C[s * k:(s + 1) * k], invn[s * 2 * k:(s + 1) * 2 * k])
+        assert torch.equal(f[s], f1) and torch.equal(alpha[s], a1)
+        # the oracle, run per projection with that projection's index set
+        rep = parity.Report(b=b, k=k)
+        C64, q = orc.gather(X, idx[s * k:(s + 1) * k].cpu().numpy())
+        f_e, a_e = parity.check_compress(X, C64, q, f[s].cpu().numpy(), alpha[s].cpu().numpy(), rep, dtype)
+        # backward per projection on its own columns of dY and dW
+        dYs = dYd[:, col:col + ms[s]]
+        Bt = pamm.contract(f[s], alpha[s], dYs, k)
+        pamm.weight_grad(C[s * k:(s + 1) * k], Bt, dW=dW[:, col:col + ms[s]])
+        ref = orc.weight_grad(C64, orc.contract(f_e, a_e, np.ascontiguousarray(dY[:, col:col + ms[s]]), k))
+        assert parity.rel_fro(dW[:, col:col + ms[s]].cpu().numpy(), ref) <= parity.TOL_TIGHT[dtype]
+        col += ms[s]
+    assert pamm.last_device_status() == pamm.OK
+
+
+def test_adapter_shaped_layer_with_a_narrow_output():
+    # the input of a low-rank adapter's first matrix (Section 4.7 applies the method there): m is the adapter's rank
+    X, dY = synth.random_case(4096, 1288, 16, "bf16", seed=81, centres=30, dy_scale=1e-3)
+    rep = parity.run_and_compare(X, dY, 32, seed=82, products=True)
+    assert rep.unexplained == 0
+    rep = parity.run_and_compare(X, dY, 32, seed=82, dw_dtype=torch.bfloat16, layout=pamm.DW_MN)
+    assert rep.unexplained == 0
 
 
 def test_contract_with_many_generators_uses_large_shared_histograms():
