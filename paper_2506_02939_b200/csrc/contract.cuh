@@ -128,11 +128,17 @@ contract_scan_kernel(int32_t* __restrict__ hist, int nb, int k, int32_t* __restr
     if (tid == 0) seg_start[k] = s_carry;
 }
 
-// Stable ranking of up to SORT_BLK rows of one block, warp by warp in ascending row
-// order: inside a warp, match_any groups equal keys and the lowest lane of a group
-// reserves the group's slots in s_next.  A slot outside [0, b) can only come from counts
-// that do not belong to this f (a caller's mistake): it is skipped and reported.
-__device__ __forceinline__ void scatter_chunk(int32_t key, int64_t i, int nrows, int32_t* s_next,
+// Stable ranking of up to SORT_BLK rows of one block in ascending row order.  Inside a
+// warp, match_any groups equal keys (rank = position inside the group, the lowest lane
+// leads).  Across the warps of the block either
+//   - a table of per-warp counts (s_tbl != nullptr: warps x k words of shared memory):
+//     the leaders post their group sizes, one thread per key turns the column of its key
+//     into running slot numbers (continuing s_next), and every row reads its slot; or
+//   - warp by warp, each leader reserving its group's slots in s_next in turn
+//     (no extra shared memory, as many block-wide barriers as there are warps).
+// A slot outside [0, b) can only come from counts that do not belong to this f (a caller's
+// mistake): it is skipped and reported.
+__device__ __forceinline__ void scatter_chunk(int32_t key, int64_t i, int nrows, int k, int32_t* s_next, int32_t* s_tbl,
                                               int32_t* __restrict__ perm, int64_t b) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned peers = __match_any_sync(0xffffffffu, key);
@@ -140,6 +146,29 @@ __device__ __forceinline__ void scatter_chunk(int32_t key, int64_t i, int nrows,
     const int leader = __ffs(peers) - 1;
     const int count = __popc(peers);
     const int warps = (nrows + 31) >> 5;
+    if (s_tbl) {
+        for (int t = threadIdx.x; t < warps * k; t += SORT_BLK) s_tbl[t] = 0;
+        __syncthreads();
+        if (lane == leader && key >= 0) s_tbl[warp * k + key] = count;
+        __syncthreads();
+        for (int j = threadIdx.x; j < k; j += SORT_BLK) {
+            int32_t run = s_next[j];
+            for (int w = 0; w < warps; ++w) {
+                const int32_t c = s_tbl[w * k + j];
+                s_tbl[w * k + j] = run;
+                run += c;
+            }
+            s_next[j] = run;
+        }
+        __syncthreads();
+        if (key >= 0) {
+            const int64_t pos = (int64_t)s_tbl[warp * k + key] + rank;
+            if (pos >= 0 && pos < b) perm[pos] = (int32_t)i;
+            else raise_status(DEV_BAD_INDEX);
+        }
+        __syncthreads();
+        return;
+    }
     for (int w = 0; w < warps; ++w) {
         __syncthreads();
         if (warp == w) {
@@ -159,12 +188,19 @@ __device__ __forceinline__ void scatter_chunk(int32_t key, int64_t i, int nrows,
     __syncthreads();
 }
 
+// Warps of a block's largest chunk, and whether their count table fits beside s_next.
+inline int scatter_table_warps(int64_t rows_per_block, int64_t k) {
+    const int warps = (int)((std::min<int64_t>(rows_per_block, SORT_BLK) + 31) / 32);
+    return (int64_t)(1 + warps) * k * 4 <= 96 * 1024 ? warps : 0;
+}
+
 // Stable scatter of one block's rows, given the scanned tables.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
+contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block, int tbl_warps,
                         const int32_t* __restrict__ hist, const int32_t* __restrict__ seg_start,
                         int32_t* __restrict__ perm) {
-    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
+    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block, then the count table
+    int32_t* s_tbl = tbl_warps ? s_next + k : nullptr;
     const int tid = threadIdx.x;
     const int32_t* my_hist = hist + (int64_t)blockIdx.x * k;
     grid_dependency_wait();
@@ -179,7 +215,7 @@ contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k
             key = load_index(f, f_type, i);
             if (key < 0 || key >= k) key = -1;
         }
-        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), s_next, perm, b);
+        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), k, s_next, s_tbl, perm, b);
     }
 }
 
@@ -193,10 +229,11 @@ contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k
 // threads: with W = the chunk's width rounded up to a power of two, the SORT_BLK
 // / W thread groups each take every (SORT_BLK / W)-th histogram row.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
+contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block, int tbl_warps,
                              const int32_t* __restrict__ hist, int nb, int32_t* __restrict__ seg_start,
                              int32_t* __restrict__ perm) {
-    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block
+    extern __shared__ int32_t s_next[];    // next free slot of every segment for this block, then the count table
+    int32_t* s_tbl = tbl_warps ? s_next + k : nullptr;
     __shared__ int32_t s_part[2][SORT_BLK];   // per-thread partial (total, before) of the column sums
     __shared__ int32_t s_warp[32];
     __shared__ int32_t s_carry;
@@ -283,7 +320,7 @@ contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, 
             key = load_index(f, f_type, i);
             if (key < 0 || key >= k) key = -1;
         }
-        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), s_next, perm, b);
+        scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), k, s_next, s_tbl, perm, b);
     }
 }
 

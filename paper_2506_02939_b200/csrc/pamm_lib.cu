@@ -188,11 +188,13 @@ constexpr int64_t FUSED_SCAN_LIMIT = 1ll << 24;
 pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const int32_t* products, const ContractWs& w,
                         cudaStream_t st) {
     const size_t hsmem = (size_t)k * 4;
-    if (!ensure_dynamic_smem((const void*)contract_hist_kernel, hsmem) ||
-        !ensure_dynamic_smem((const void*)contract_scatter_kernel, hsmem) ||
-        !ensure_dynamic_smem((const void*)contract_scan_scatter_kernel, hsmem))
-        return PAMM_ERR_CUDA;
     const int rpb = (int)w.rows_per_block;
+    const int tbl_warps = scatter_table_warps(rpb, k);
+    const size_t ssmem = (size_t)(1 + tbl_warps) * k * 4;
+    if (!ensure_dynamic_smem((const void*)contract_hist_kernel, hsmem) ||
+        !ensure_dynamic_smem((const void*)contract_scatter_kernel, ssmem) ||
+        !ensure_dynamic_smem((const void*)contract_scan_scatter_kernel, ssmem))
+        return PAMM_ERR_CUDA;
     const bool fused_scan = w.nb * w.nb * k <= FUSED_SCAN_LIMIT;
     const int32_t* hist = w.hist;
     if (products && fused_scan) {
@@ -204,12 +206,12 @@ pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const i
         launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb, w.hist);
     }
     if (fused_scan) {
-        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb,
-               hist, (int)w.nb, w.seg_start, w.perm);
+        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, b, (int)k, rpb,
+               tbl_warps, hist, (int)w.nb, w.seg_start, w.perm);
     } else {
         launch(contract_scan_kernel, dim3(1), dim3(SCAN_THREADS), 0, st, true, w.hist, (int)w.nb, (int)k, w.seg_start);
-        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb,
-               (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
+        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, b, (int)k, rpb,
+               tbl_warps, (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
     }
     return launch_status();
 }

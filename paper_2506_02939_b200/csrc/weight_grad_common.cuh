@@ -68,6 +68,40 @@ __device__ __forceinline__ void load_bt8(const float* __restrict__ Bt, int64_t l
     }
 }
 
+// Converts the 128-column block of B~ that starts at column m0 (kc generator rows, zero rows
+// past k) into the bf16 hi / lo operand blocks, with `nth` threads of which the caller is
+// number `t` (whole warps, t - lane a multiple of 32).  Items (one generator x 8 columns)
+// are dealt round-robin, so a warp's 32 items always lie in one group of 16 generators;
+// BATCH rounds of loads are in flight together, and after every round each warp announces
+// its share on the group's barrier (eight warp-arrivals complete a group).
+template <int BATCH>
+__device__ __forceinline__ void convert_bt_block(const float* __restrict__ Bt, int64_t ldb, int k, int64_t m, int kc,
+                                                 int64_t m0, uint8_t* sBhi, uint8_t* sBlo, uint32_t blk_bytes,
+                                                 uint64_t* s_bfull, int t, int nth) {
+    const int items = kc * 16;
+    const bool full_cols = m0 + WG_TILE <= m;
+    const int lane = threadIdx.x & 31;
+    for (int base = 0; base < items; base += BATCH * nth) {
+        float4 a4[BATCH], b4[BATCH];
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {     // every load of the batch first
+            const int idx = base + u * nth + t;
+            a4[u] = b4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (idx < items && (idx >> 4) < k) load_bt8(Bt, ldb, idx >> 4, m0 + (idx & 15) * 8, m, full_cols, a4[u], b4[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const int idx = base + u * nth + t;
+            if (idx - lane < items) {         // warp-uniform: items is a multiple of 256
+                split_store_hi_lo(sBhi, sBlo, blk_bytes, idx >> 4, idx & 15, a4[u], b4[u]);
+                ptx::fence_proxy_async();     // generic-proxy stores -> visible to the tensor core's async proxy
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&s_bfull[idx >> 8]);
+            }
+        }
+    }
+}
+
 // Staging of the output tile in shared memory: TMA boxes of 128 rows x 128 bytes
 // (32 fp32 or 64 bf16 columns) in the 128-byte swizzle.  A column half of the tile
 // (64 columns) is two fp32 boxes or one bf16 box.

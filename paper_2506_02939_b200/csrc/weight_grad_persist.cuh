@@ -15,9 +15,10 @@
 //                column half share one staging area and one store stream
 //   warps 10-13  split the fp32 B~ column block into bf16 hi + lo (hi = rn(x),
 //                lo = rn(x - hi), about 16 mantissa bits together) in the MN-major
-//                swizzled operand layout, once per column block; the loads of 64 generators
-//                are in flight at once and every group of 16 generators is announced
-//                on its own barrier
+//                swizzled operand layout, once per column block; every group of 16
+//                generators is announced on its own barrier.  The CTA's FIRST block is
+//                converted by these warps and the eight epilogue warps together: nothing
+//                can be stored before it exists, so they would only wait
 // (fourteen warps: four per scheduler at most, which leaves each thread 128 registers)
 // When there are at least as many SMs as column blocks, every column block is
 // shared by a fixed number of CTAs that split its row tiles, so no CTA ever
@@ -78,7 +79,7 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
             ptx::mbar_init(&s_tfull[s], 1);
             ptx::mbar_init(&s_tempty[s], WG_EPI_WARPS);
         }
-        for (int g = 0; g < WP_MAX_GROUPS; ++g) ptx::mbar_init(&s_bfull[g], WP_CVT_THREADS / 32);
+        for (int g = 0; g < WP_MAX_GROUPS; ++g) ptx::mbar_init(&s_bfull[g], 8);   // 256 items of 32 per warp-arrival
         ptx::mbar_init(&s_bempty, 1);
         s_abort = 0;
         ptx::fence_barrier_init();
@@ -163,6 +164,9 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
         }
     } else if (warp < 2 + WG_EPI_WARPS) {
         // ---------------- epilogue: 32 rows x 64 columns of the tile per warp ----------------
+        if (t0 < t1)      // lend a hand with the first B~ block
+            convert_bt_block<6>(Bt, ldb, k, m, kc, (int64_t)(t0 / n_tiles) * WG_TILE, sBhi, sBlo, blk_bytes, s_bfull, tid - 64,
+                                WP_THREADS - 64);
         const int quad = warp & 3;                       // TMEM lanes [32*quad, 32*quad+32)
         const int h = (warp - 2) >> 2;                   // column half
         const bool leader = ((warp - 2) & 3) == 0 && lane == 0;
@@ -182,9 +186,6 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
         if (!ok && lane == 0) raise_status(DEV_TIMEOUT);
     } else {
         // ---------------- B~ column block: fp32 -> bf16 hi / lo, swizzled MN-major ----------------
-        const int ctid = tid - WP_CVT_TID0;
-        const int jr0 = ctid >> 4, cg = ctid & 15;       // my two generators of a group of 16 (jr0, jr0 + 8), my 8-column group
-        constexpr int BATCH = 4;                         // generator groups whose loads are in flight together
         uint32_t g = 0;
         int prev_cb = -1;
         bool ok = true;
@@ -192,34 +193,14 @@ weight_grad_persist_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
             const int cb = t / n_tiles;
             if (cb == prev_cb) continue;
             prev_cb = cb;
-            if (g > 0) {
+            if (g == 0) {     // the first block, together with the epilogue warps
+                convert_bt_block<6>(Bt, ldb, k, m, kc, (int64_t)cb * WG_TILE, sBhi, sBlo, blk_bytes, s_bfull, tid - 64,
+                                    WP_THREADS - 64);
+            } else {
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_bempty, (g - 1) & 1u, abort_flag));
                 if (!ok) break;
-            }
-            const int64_t m0 = (int64_t)cb * WG_TILE;
-            const int64_t col = m0 + cg * 8;
-            const bool full_cols = m0 + WG_TILE <= m;
-            for (int u0 = 0; u0 < groups; u0 += BATCH) {
-                float4 a4[BATCH][2], b4[BATCH][2];
-#pragma unroll
-                for (int u = 0; u < BATCH; ++u)          // every load of the batch first
-#pragma unroll
-                    for (int v = 0; v < 2; ++v) {
-                        a4[u][v] = b4[u][v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        const int jr = (u0 + u) * 16 + jr0 + 8 * v;
-                        if (u0 + u < groups && jr < k) load_bt8(Bt, ldb, jr, col, m, full_cols, a4[u][v], b4[u][v]);
-                    }
-#pragma unroll
-                for (int u = 0; u < BATCH; ++u) {
-                    if (u0 + u < groups) {
-#pragma unroll
-                        for (int v = 0; v < 2; ++v)
-                            split_store_hi_lo(sBhi, sBlo, blk_bytes, (u0 + u) * 16 + jr0 + 8 * v, cg, a4[u][v], b4[u][v]);
-                        ptx::fence_proxy_async();    // generic-proxy stores -> visible to the tensor core's async proxy
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&s_bfull[u0 + u]);
-                    }
-                }
+                convert_bt_block<4>(Bt, ldb, k, m, kc, (int64_t)cb * WG_TILE, sBhi, sBlo, blk_bytes, s_bfull,
+                                    tid - WP_CVT_TID0, WP_CVT_THREADS);
             }
             ++g;
         }
