@@ -32,7 +32,9 @@
  * the Frobenius error bound of Section 3.2.1, and the printed gamma ~ 28; for the
  * neighbourhood condition: the equivalent cosine form csim^2 >= 1 - eps^2, eps = 0
  * against the uniform column-row-sampling estimator, eps >= 1 against eps = infinity,
- * and the exact unbiasedness of the k = 1, eps = 0 estimate averaged over all rows.
+ * and the exact unbiasedness of the k = 1, eps = 0 estimate averaged over all rows; for
+ * the layer's output Z = X W (Algorithm 2): a 2 x 2 product worked by hand, numpy's matmul,
+ * and the identity that X C^T reproduces the dot products behind f and alpha.
  */
 #include <math.h>
 #include <stdint.h>
@@ -223,6 +225,27 @@ void pamm_oracle_exact_product(const void *A, int dtypeA, int64_t lda, const voi
             for (int64_t i = 0; i < b; ++i)
                 acc += widen(A, dtypeA, i * lda + r) * widen(B, dtypeB, i * ldb + c);
             O_out[r * m + c] = acc;
+        }
+    }
+}
+
+/* Algorithm 2 (forward pass of the linear layer), first step: Z = X W, the layer's output,
+ * computed from the same X that Compress then reduces to (C, alpha, f).  X is b x n, W is
+ * n x m (the paper's orientation: Z_ic = sum_l X_il W_lc), Z is b x m.  A plain triple
+ * loop; `rows` (may be NULL) restricts the computation to the listed rows of X, whose
+ * results are written to the first nrows rows of Z_out. */
+void pamm_oracle_linear_forward(const void *X, int dtypeX, int64_t ldx, const void *W, int dtypeW, int64_t ldw,
+                                int64_t b, int64_t n, int64_t m, const int64_t *rows, int64_t nrows, double *Z_out)
+{
+    int64_t count = rows ? nrows : b, t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < count; ++t) {
+        int64_t i = rows ? rows[t] : t;
+        for (int64_t c = 0; c < m; ++c) {
+            double acc = 0.0;
+            for (int64_t l = 0; l < n; ++l)
+                acc += widen(X, dtypeX, i * ldx + l) * widen(W, dtypeW, l * ldw + c);
+            Z_out[t * m + c] = acc;
         }
     }
 }

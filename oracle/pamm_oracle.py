@@ -63,6 +63,8 @@ def _load():
         L.pamm_oracle_beta.restype = ctypes.c_double
         L.pamm_oracle_exact_product.argtypes = [vp, ci, i64, vp, ci, i64, i64, i64, i64, vp]
         L.pamm_oracle_exact_product.restype = None
+        L.pamm_oracle_linear_forward.argtypes = [vp, ci, i64, vp, ci, i64, i64, i64, i64, vp, i64, vp]
+        L.pamm_oracle_linear_forward.restype = None
         L.pamm_oracle_memory_scalars.argtypes = [i64, i64, i64]
         L.pamm_oracle_memory_scalars.restype = i64
         L.pamm_oracle_gamma.argtypes = [i64, i64, i64]
@@ -203,6 +205,25 @@ def exact_product(A: np.ndarray, B: np.ndarray) -> np.ndarray:
     O = np.empty((n, m), np.float64)
     _load().pamm_oracle_exact_product(_p(A), _dtype_code(A), _ld(A), _p(B), _dtype_code(B), _ld(B), b, n, m, _p(O))
     return O
+
+
+def linear_forward(X: np.ndarray, W: np.ndarray, rows=None) -> np.ndarray:
+    """Z = X W (Algorithm 2, the layer's output), optionally for the listed rows of X only."""
+    X, W = _mat(X), _mat(W)
+    b, n = X.shape
+    m = W.shape[1]
+    assert W.shape[0] == n
+    if rows is None:
+        Z = np.empty((b, m), np.float64)
+        _load().pamm_oracle_linear_forward(_p(X), _dtype_code(X), _ld(X), _p(W), _dtype_code(W), _ld(W), b, n, m,
+                                           None, 0, _p(Z))
+        return Z
+    rows = np.ascontiguousarray(rows, np.int64)
+    assert rows.min() >= 0 and rows.max() < b
+    Z = np.empty((rows.size, m), np.float64)
+    _load().pamm_oracle_linear_forward(_p(X), _dtype_code(X), _ld(X), _p(W), _dtype_code(W), _ld(W), b, n, m,
+                                       _p(rows), rows.size, _p(Z))
+    return Z
 
 
 def memory_scalars(b: int, n: int, k: int) -> int:

@@ -383,3 +383,43 @@ def test_kept_set_grows_with_epsilon_and_error_bound_holds():
         lhs = np.linalg.norm(X64.T @ B - r["O"] / r["beta"], "fro") ** 2
         rhs = np.linalg.norm(B, 2) ** 2 * (eps ** 2 * np.sum(X64[r["kept"]] ** 2) + np.sum(X64[~r["kept"]] ** 2))
         assert lhs <= rhs * (1 + 1e-12) + 1e-18
+
+
+# ---- Algorithm 2, first step: the layer's output Z = X W ---------------------------------
+
+def test_linear_forward_hand_computed_two_by_two():
+    # [[1, 2], [3, 4]] [[5, 6], [7, 8]] = [[19, 22], [43, 50]], worked by hand
+    X = np.array([[1, 2], [3, 4]], np.float32)
+    W = np.array([[5, 6], [7, 8]], np.float32)
+    assert np.array_equal(orc.linear_forward(X, W), np.array([[19.0, 22.0], [43.0, 50.0]]))
+    # not its transpose-side variants: W X, X^T W, X W^T all differ on this example
+    assert not np.array_equal(orc.linear_forward(X, W), (W @ X).astype(np.float64))
+    assert not np.array_equal(orc.linear_forward(X, W), (X.T @ W).astype(np.float64))
+    assert not np.array_equal(orc.linear_forward(X, W), (X @ W.T).astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_linear_forward_is_the_plain_matrix_product(dtype):
+    X, _ = synth.random_case(37, 29, 8, dtype, seed=3)
+    W, _ = synth.random_case(29, 23, 8, dtype, seed=4)
+    Z = orc.linear_forward(X, W)
+    ref = synth.to_f64(X) @ synth.to_f64(W)
+    assert Z.shape == (37, 23) and np.allclose(Z, ref, rtol=1e-13, atol=1e-13)
+    rows = np.array([5, 0, 36, 5])
+    assert np.array_equal(orc.linear_forward(X, W, rows=rows), Z[rows])
+    # a padded row stride of either operand changes nothing
+    Xp = np.zeros((37, 40), X.dtype); Xp[:, :29] = X
+    Wp = np.zeros((29, 32), W.dtype); Wp[:, :23] = W
+    assert np.array_equal(orc.linear_forward(Xp[:, :29], Wp[:, :23]), Z)
+
+
+def test_linear_forward_and_compress_see_the_same_input():
+    # Algorithm 2: Z = X W and Compress(X) come from the same X.  The scores are the extra columns of X [W | C^T]:
+    # the forward product against C^T reproduces the dot products behind f and alpha (Eq. 1)
+    X, _ = synth.random_case(64, 24, 8, "bf16", seed=9, centres=5)
+    I = np.array([3, 17, 40], np.int32)
+    C64, q = orc.gather(X, I)
+    f, alpha, _, _ = orc.compress(X, C64, q)
+    S = orc.linear_forward(X, np.ascontiguousarray(X[I].T))          # b x k: X C^T
+    assert np.array_equal(np.argmax(np.abs(S) / np.sqrt(q), axis=1), f)
+    assert np.allclose(S[np.arange(64), f] / q[f], alpha, rtol=1e-14, atol=0)
