@@ -147,6 +147,31 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
                                 void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * The forward pass of the linear layer with the compression fused into it (Algorithm 2:
+ * Z = X W; (C, alpha, f) = Compress(flatten(X)); keep C, alpha, f instead of X).  The
+ * scores X C^T are k more output columns of the product X [W | C^T]: ONE tensor-core
+ * kernel computes Z and, from the row blocks of X it has in flight anyway, f and alpha,
+ * so the compression costs no pass over X of its own.  Generators are drawn (or taken
+ * from idx_in) as in pamm_compress_fused; f, alpha and the sort products are bit for bit
+ * those of pamm_compress_fused.
+ *   X  b x n   W  n x m (Z_ic = sum_l X_il W_lc)   Z  b x m, all of dtype dt, row-major
+ *   dt  PAMM_BF16 only (fp32 accumulation, Z rounded to nearest even); anything else, or
+ *       0 < k < 16 or k > 4096, returns PAMM_ERR_UNSUPPORTED -- there is no other
+ *       implementation behind this call
+ *   k   0 computes Z alone (a layer whose input needs no gradient, or evaluation): the
+ *       compression arguments are then ignored and may be NULL
+ * X and W must be complete when the call is enqueued in the sense of every other call
+ * (work enqueued earlier on the stream has produced them).
+ */
+pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n,
+                                const void* W, int64_t ldw, int64_t m, pamm_dtype dt,
+                                int64_t k, uint64_t seed, const int32_t* idx_in,
+                                int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
+                                void* Z, int64_t ldz,
+                                void* f, pamm_index_type f_type, float* alpha,
+                                void* workspace, size_t ws_bytes, void* stream);
+
+/*
  * Step 2 for several generator sets at once -- one compression per projection
  * (Section 4: the method "is applied to the Q, K and V projections"; the worked
  * example of the appendix "Complexity Analysis" has m = n per projection) -- in ONE

@@ -18,6 +18,7 @@
 #include "weight_grad_simt.cuh"
 #include "weight_grad_persist.cuh"
 #include "weight_grad_chunked.cuh"
+#include "linear_forward.cuh"
 
 using namespace pamm;
 
@@ -144,13 +145,13 @@ StepArena step_arena_layout(void* base, int64_t b, int64_t n, int64_t m, int64_t
 template <typename T>
 pamm_status launch_select(const void* X, int64_t ldx, int64_t b, int64_t n, int64_t k, uint64_t seed,
                           const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
-                          cudaStream_t st) {
+                          cudaStream_t st, int32_t* zero_words = nullptr, int64_t zero_count = 0) {
     const size_t smem = (size_t)k * 4;
     if (!ensure_dynamic_smem((const void*)select_kernel<T>, smem)) return PAMM_ERR_CUDA;
     const PermKey pk = make_perm_key(seed, (uint32_t)b);
     const int grid = (int)k;
     launch(select_kernel<T>, dim3(grid), dim3(SEL_THREADS), smem, st, true, (const T*)X, ldx, b, n, (int)k, pk, idx_in,
-           idx_out, (T*)C, ldc, c_invnorm);
+           idx_out, (T*)C, ldc, c_invnorm, zero_words, zero_count);
     return launch_status();
 }
 
@@ -553,6 +554,43 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
                        : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
     if (s != PAMM_OK) return s;
     return do_compress(X, ldx, b, n, dt, C, ldc, k, 1, c_invnorm, f, f_type, alpha, b, (int32_t*)workspace, true, st);
+}
+
+pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n, const void* W, int64_t ldw, int64_t m,
+                                pamm_dtype dt, int64_t k, uint64_t seed, const int32_t* idx_in, int32_t* idx_out,
+                                void* C, int64_t ldc, float* c_invnorm, void* Z, int64_t ldz, void* f,
+                                pamm_index_type f_type, float* alpha, void* workspace, size_t ws_bytes, void* stream) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!X || !W || !Z || b < 1 || n < 1 || m < 1 || k < 0 || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(ldx, n, esize(dt)) || !ld_ok(ldw, m, esize(dt)) || !ld_ok(ldz, m, esize(dt))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(X, 16) || !aligned(W, 16) || !aligned(Z, 16)) return PAMM_ERR_INVALID_ARG;
+    pamm_status s = PAMM_OK;
+    if (k > 0) {
+        s = check_select(X, ldx, b, n, dt, k, idx_out, C, ldc, c_invnorm);
+        if (s != PAMM_OK) return s;
+        s = check_compress(X, ldx, b, n, dt, C, ldc, k, c_invnorm, f, f_type, alpha);
+        if (s != PAMM_OK) return s;
+        s = check_products_out(workspace, ws_bytes, b, k, 1);
+        if (s != PAMM_OK) return s;
+    }
+    // the tensor-core kernel is the only implementation: no CUDA-core or library GEMM stands in for it
+    if (dt != PAMM_BF16 || !linear_forward_supported(b, n, m, k) ||
+        linear_forward_plan_for(b, m, k, sm_count()).stages < 2)
+        return PAMM_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t rpb = sort_rows_per_block(b);
+    int32_t* hist = k > 0 ? (int32_t*)workspace : nullptr;
+    if (k > 0) {
+        s = launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st, hist,
+                                         hist ? ((b + rpb - 1) / rpb) * k : 0);
+        if (s != PAMM_OK) return s;
+    }
+    const LinearForwardOut out = {f, alpha, hist, (int)rpb, (int)f_type};
+    prof_begin(PAMM_PROF_COMPRESS, st);
+    s = launch_linear_forward(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st);
+    prof_end(PAMM_PROF_COMPRESS, st);
+    g_launches += 1;
+    return s;
 }
 
 pamm_status pamm_contract(const void* f, pamm_index_type f_type, const float* alpha, const void* dY, int64_t ldy,

@@ -27,7 +27,8 @@ template <typename T>
 __global__ void __launch_bounds__(SEL_THREADS)
 select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k, PermKey pk,
               const int32_t* __restrict__ idx_in, int32_t* __restrict__ idx_out,
-              T* __restrict__ C, int64_t ldc, float* __restrict__ c_invnorm) {
+              T* __restrict__ C, int64_t ldc, float* __restrict__ c_invnorm,
+              int32_t* __restrict__ zero_words, int64_t zero_count) {
     extern __shared__ int32_t s_vals[];
     __shared__ int s_cnt[2][SEL_WARPS];
     __shared__ float s_q[2][SEL_WARPS];
@@ -41,6 +42,9 @@ select_kernel(const T* __restrict__ X, int64_t ldx, int64_t b, int64_t n, int k,
     grid_launch_dependents();
     if (idx_in)
         for (int j = tid; j < k; j += SEL_THREADS) s_vals[j] = idx_in[j];
+    // counters the next kernel adds to (the histograms of f of the fused forward pass) start at zero
+    for (int64_t z = (int64_t)blockIdx.x * SEL_THREADS + tid; z < zero_count; z += (int64_t)gridDim.x * SEL_THREADS)
+        zero_words[z] = 0;
     __syncthreads();
 
     const int j = blockIdx.x;          // one CTA per generator

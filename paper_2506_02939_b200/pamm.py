@@ -37,6 +37,8 @@ _SIGNATURES = {
     "pamm_compress": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _vp, _ci, _vp, _vp, _sz, _vp], _ci),
     "pamm_compress_fused": ([_vp, _i64, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _ci, _vp, _vp, _sz, _vp], _ci),
     "pamm_compress_projections": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _ci, _vp, _i64, _vp, _sz, _vp], _ci),
+    "pamm_linear_forward": ([_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _vp, _ci,
+                             _vp, _vp, _sz, _vp], _ci),
     "pamm_contract": ([_vp, _ci, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _vp, _sz, _vp], _ci),
     "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _ci, _ci, _vp], _ci),
     "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _ci, _vp, _vp, _vp, _sz, _vp], _ci),
@@ -243,6 +245,24 @@ def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, 
                                     _ld(C), _ptr(c_invnorm), _ptr(f), _ft(f), _ptr(alpha), _ptr(sort_products),
                                     _bytes(sort_products), _stream(stream)), "pamm_compress_fused")
     return idx_out, C, c_invnorm, f, alpha
+
+
+def linear_forward(X, W, k: int, seed: int = 0, idx_in=None, Z=None, idx_out=None, C=None, c_invnorm=None, f=None, alpha=None,
+                   sort_products=None, f_dtype=None, stream=None):
+    """Algorithm 2 in one tensor-core kernel: ``Z = X W`` (W is n x m) and the compression of X.  bf16 only."""
+    b, n = X.shape
+    m = W.shape[1]
+    dev = X.device
+    Z = alloc_matrix(b, m, X.dtype, dev) if Z is None else Z
+    idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
+    C = alloc_matrix(k, n, X.dtype, dev) if C is None else C
+    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
+    f = _new_f(b, f_dtype, dev) if f is None else f
+    alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
+    _check(_lib.pamm_linear_forward(_ptr(X), _ld(X), b, n, _ptr(W), _ld(W), m, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out),
+                                    _ptr(C), _ld(C), _ptr(c_invnorm), _ptr(Z), _ld(Z), _ptr(f), _ft(f), _ptr(alpha),
+                                    _ptr(sort_products), _bytes(sort_products), _stream(stream)), "pamm_linear_forward")
+    return Z, idx_out, C, c_invnorm, f, alpha
 
 
 def contract(f, alpha, dY, k: int, Btilde=None, sort_products=None, workspace=None, stream=None):
