@@ -342,6 +342,23 @@ def run_cuda(args):
         step(w.index_seed + extra)
         extra += 1
     torch.cuda.synchronize()
+
+    # each stage repeated back to back (untimed region): its throughput when the launches overlap as they do
+    # inside a step, without the event records that bracket a single stage above
+    def repeat_ms(fn, reps=64):
+        for s in range(4):
+            fn(w.index_seed + s)
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for s in range(reps):
+            fn(w.index_seed + s)
+        z.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / reps
+
+    fwd_rep = repeat_ms(forward)
+    bwd_rep = repeat_ms(lambda s: backward())
+    forward(w.index_seed)          # leave (C, f, alpha) of a forward pass behind, as after a step
     covers = "timed region"
     if t_begin.elapsed_time(t_end) < 500.0:
         # a region this short yields too few 50 ms samples: keep sampling over an untimed repeat of the same steps
@@ -405,6 +422,8 @@ def run_cuda(args):
         "compress_stage_best": frac(ab["compress"] / (st_f["min"] * 1e-3) / 1e9),
         "contract_wgrad_stage": frac((ab["contract"] + ab["weight_grad"]) / (st_b["median"] * 1e-3) / 1e9),
         "contract_wgrad_stage_best": frac((ab["contract"] + ab["weight_grad"]) / (st_b["min"] * 1e-3) / 1e9),
+        "compress_stage_repeated_back_to_back": dict(ms=fwd_rep, **frac(ab["compress"] / (fwd_rep * 1e-3) / 1e9)),
+        "contract_wgrad_stage_repeated_back_to_back": dict(ms=bwd_rep, **frac((ab["contract"] + ab["weight_grad"]) / (bwd_rep * 1e-3) / 1e9)),
         "whole_step": frac(sum(ab.values()) / (ms_total / K * 1e-3) / 1e9),
         "kernel_ms": st_k,
         "kernel": {"compress": frac(ab["compress"] / (st_k["compress"]["median"] * 1e-3) / 1e9),
@@ -468,6 +487,96 @@ def run_cuda(args):
         "clocks": clocks,
         "stages": stages,
         "memory_saved": saved,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_forward(args):
+    """The forward pass of the layer (Algorithm 2) with the compression fused into the product:
+    time of pamm_linear_forward against the same kernel without generators plus the stand-alone
+    compression, and the tensor roofline fraction.  torch's own GEMM is timed as context only."""
+    import torch
+    from paper_2506_02939_b200 import build as pamm_build, synth
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the PAMM path has no CPU fallback")
+    torch.cuda.set_device(env_int("LOCAL_RANK", 0))
+    pamm_build.build()
+    from paper_2506_02939_b200 import pamm
+    w = synth.WORKLOADS[args.workload]
+    if w.dtype != "bf16":
+        raise SystemExit("the fused forward pass is a bf16 tensor-core kernel")
+    k = args.k or w.ks[0]
+    inp = synth.make_inputs(args.workload, with_dY=False)
+    b, n, m = inp.b, w.n, w.m
+    X = torch.from_numpy(inp.X.view(np.int16)).view(torch.bfloat16).cuda()
+    rng = np.random.default_rng([w.seed, 5])
+    W = torch.from_numpy(synth.f32_to_bf16_bits(rng.standard_normal((n, m), dtype=np.float32) / np.float32(np.sqrt(n)))
+                         .view(np.int16)).view(torch.bfloat16).cuda()
+    dev = X.device
+    Z = torch.empty((b, m), dtype=torch.bfloat16, device=dev)
+    idx = torch.empty(k, dtype=torch.int32, device=dev)
+    C = torch.empty((k, n), dtype=torch.bfloat16, device=dev)
+    invn = torch.empty(2 * k, dtype=torch.float32, device=dev)
+    f = torch.empty(b, dtype=torch.int32, device=dev)
+    alpha = torch.empty(b, dtype=torch.float32, device=dev)
+    sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, pamm.BF16, dev)
+    stream = torch.cuda.current_stream()
+
+    def fused(s):
+        pamm.linear_forward(X, W, k, w.index_seed + s, Z=Z, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha,
+                            sort_products=sp, stream=stream)
+
+    def product_alone(s):
+        pamm.linear_forward(X, W, 0, Z=Z, stream=stream)
+
+    def compress_alone(s):
+        pamm.compress_fused(X, k, w.index_seed + s, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, sort_products=sp,
+                            stream=stream)
+
+    def torch_gemm(s):
+        torch.matmul(X, W, out=Z)
+
+    def timed(fn, steps):
+        for s in range(3):
+            fn(s)
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record(stream)
+        for s in range(steps):
+            fn(s)
+            ev[s + 1].record(stream)
+        torch.cuda.synchronize()
+        return stats([ev[s].elapsed_time(ev[s + 1]) for s in range(steps)])
+
+    K = max(5, min(args.steps, 50))
+    sampler = ClockSampler(env_int("LOCAL_RANK", 0))
+    sampler.start()
+    launches0 = pamm.launch_count()
+    t_fused = timed(fused, K)
+    launches = pamm.launch_count() - launches0
+    t_prod = timed(product_alone, K)
+    t_comp = timed(compress_alone, K)
+    t_torch = timed(torch_gemm, K)
+    clocks = sampler.stop()
+    status = pamm.last_device_status()
+    if status != pamm.OK:
+        raise SystemExit(f"device status: {pamm.status_string(status)}")
+    peak, peak_tf, peak_kind = measured_peaks()
+    flops = 2.0 * b * n * (m + k)
+    tf = flops / (t_fused["median"] * 1e-3) / 1e12
+    line = {
+        "metric": "fused forward pass Z = X W with Compress(X): tokens/s per QKV layer", "value": b / (t_fused["median"] * 1e-3),
+        "unit": "tokens/s", "n_gpus": 1, "steps": K, "warmup": 3, "ms_per_step": t_fused["median"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name} forward: X bf16 b={b} n={n}, W n x m={m}, k={k}", "l2": "inputs exceed L2"},
+        "roofline": {"bound": "tensor", "kernel": "linear_forward_kernel (X [W | C^T], 128 x 256 tiles)", "achieved": tf,
+                     "peak": peak_tf, "peak_source": f"of {peak_kind} (sustained bf16)", "unit": "TFLOP/s", "frac": tf / peak_tf,
+                     "traffic": None, "algorithmic_flops": flops},
+        "forward_ms": {"fused_product_and_compression": t_fused, "product_alone_same_kernel": t_prod,
+                       "compression_alone": t_comp,
+                       "cost_of_compression_inside_the_product_ms": t_fused["median"] - t_prod["median"],
+                       "torch_matmul_context_only": t_torch},
+        "gpu_launches": int(launches), "clocks": clocks,
     }
     print(json.dumps(line), flush=True)
 
@@ -569,6 +678,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--eps", type=float, default=None,
                     help="time the neighbourhood-condition path (Eq. 2, beta) with this epsilon instead of epsilon = infinity")
+    ap.add_argument("--forward", action="store_true",
+                    help="time the layer's forward pass with the compression fused into the product (Algorithm 2) instead")
     ap.add_argument("--dw-dtype", choices=["f32", "bf16"], default="f32", help="storage type of the weight gradient")
     ap.add_argument("--layout", choices=["nm", "mn"], default="nm", help="dW as n x m (the paper's) or m x n (out x in)")
     ap.add_argument("--layers", type=int, default=1,
@@ -583,6 +694,8 @@ def main():
         args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
+    elif args.forward:
+        run_forward(args)
     elif args.layers > 1:
         run_layer_loop(args)
     else:

@@ -1,9 +1,11 @@
 """A linear layer whose backward pass keeps the compressed input only (Algorithms 2 and 3).
 
-Forward: ``Z = X W`` (an ordinary GEMM, done by torch) and ``Compress(flatten(X))`` through
-the CUDA library; the layer saves (C, f, alpha, W) and lets go of X.  Backward: the weight
-gradient is ``ApproxMM(C, alpha, f, dZ) = C^T B~`` through the library, the input gradient
-``dX = dZ W^T`` is exact (torch).  Meant for the fused Q|K|V projection: ``W`` is n x m
+Forward: ``Z = X W`` and ``Compress(flatten(X))``.  For bf16 layers both come out of ONE kernel
+of the CUDA library (``pamm_linear_forward``: the scores are extra output columns of the
+product, so X is not read a second time); other dtypes take torch's GEMM for Z and the
+library's stand-alone compression.  The layer saves (C, f, alpha, W) and lets go of X.
+Backward: the weight gradient is ``ApproxMM(C, alpha, f, dZ) = C^T B~`` through the library,
+the input gradient ``dX = dZ W^T`` is exact (torch).  Meant for the fused Q|K|V projection: ``W`` is n x m
 with m = |Q| + |K| + |V|, as in the paper's notation.
 """
 from __future__ import annotations
@@ -29,14 +31,21 @@ class PammLinearFunction(torch.autograd.Function):
     @staticmethod
     def forward(ctx, X, W, k, seed):
         n, m = W.shape
-        Z = X @ W
         X2 = _rows(X.detach(), n)
         b = X2.shape[0]
         f_dtype = torch.uint8 if k <= 256 else torch.int16 if k <= 65536 else torch.int32
         # the pass also leaves its per-block counts of f (a few KiB): the backward's counting sort starts from them
         sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, int(k), pamm.BF16 if X2.dtype == torch.bfloat16 else pamm.F32,
                                   X2.device)
-        _, C, _, f, alpha = pamm.compress_fused(X2, int(k), int(seed), sort_products=sp, f_dtype=f_dtype)
+        Wd = W.detach()
+        one_kernel = (X2.dtype == torch.bfloat16 and Wd.dtype == torch.bfloat16 and 16 <= k <= 4096 and n >= 8 and m >= 8
+                      and Wd.is_contiguous() and (m * 2) % 16 == 0 and Wd.data_ptr() % 16 == 0)
+        if one_kernel:
+            Z2, _, C, _, f, alpha = pamm.linear_forward(X2, Wd, int(k), int(seed), sort_products=sp, f_dtype=f_dtype)
+            Z = Z2.reshape(*X.shape[:-1], m)
+        else:
+            Z = X @ W
+            _, C, _, f, alpha = pamm.compress_fused(X2, int(k), int(seed), sort_products=sp, f_dtype=f_dtype)
         ctx.save_for_backward(C, f, alpha, sp, W)      # k n + 2 b scalars instead of b n
         return Z
 
