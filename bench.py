@@ -256,17 +256,24 @@ def run_cuda(args):
     eps = args.eps
     dropped = torch.zeros(1, dtype=torch.int32, device=dev)
 
+    # the arguments of the two fused calls are marshalled once (a fresh index seed per step, 64 of them in turn):
+    # at the small workloads a step is a few microseconds of GPU work and Python's argument handling would dominate
+    SEEDS = 64
+    fwd_calls = [pamm.prepared(pamm.compress_fused, X, k, w.index_seed + s, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha,
+                               sort_products=sp, stream=stream) for s in range(SEEDS)] if eps is None else None
+    bwd_call = pamm.prepared(pamm.contract_weight_grad, C, f, alpha, dY, Btilde=Bt, dW=dW, layout=layout, sort_products=sp,
+                             workspace=ws, stream=stream) if eps is None else None
+
     def forward(seed):
         if eps is None:
-            pamm.compress_fused(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, sort_products=sp, stream=stream)
+            fwd_calls[(seed - w.index_seed) % SEEDS]()
         else:     # neighbourhood condition (Eq. 2): select, then compress with the row-norm warps
             pamm.select_generators(X, k, seed, idx_out=idx, C=C, c_invnorm=invn, stream=stream)
             pamm.compress_eps(X, C, invn, eps, f=f, alpha=alpha, dropped=dropped, sort_products=sp, stream=stream)
 
     def backward():
         if eps is None:
-            pamm.contract_weight_grad(C, f, alpha, dY, Btilde=Bt, dW=dW, layout=layout, sort_products=sp, workspace=ws,
-                                      stream=stream)
+            bwd_call()
         else:     # beta = b / (b - eta) applied by the product's epilogue (Eq. 4-5)
             pamm.contract(f, alpha, dY, k, Btilde=Bt, sort_products=sp, workspace=ws, stream=stream)
             pamm.weight_grad_beta(C, Bt, b, dropped, dW=dW, layout=layout, stream=stream)

@@ -129,7 +129,9 @@ pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_
  *          generator, counted on the fly by the pass.  They are an optional by-product
  *          for the backward pass (pamm_contract, pamm_contract_weight_grad), which then
  *          skips its own counting launch; they must be kept next to f until then and
- *          are valid only for this f on a device with the same number of SMs.
+ *          are valid only for this f on a device with the same number of SMs.  With
+ *          k <= 8 the backward pass does not sort at all: the argument is then ignored by
+ *          both sides and the buffer may be left untouched.
  */
 pamm_status pamm_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_dtype dt,
                           const void* C, int64_t ldc, int64_t k, const float* c_invnorm,

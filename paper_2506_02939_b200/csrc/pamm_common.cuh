@@ -105,6 +105,40 @@ __device__ __forceinline__ void load_vec<__nv_bfloat16>(const __nv_bfloat16* row
     }
 }
 
+// 16 bytes already in a register -> floats
+template <typename T>
+__device__ __forceinline__ void unpack_vec(const uint4& raw, float (&out)[Vec16<T>::N]);
+template <>
+__device__ __forceinline__ void unpack_vec<float>(const uint4& raw, float (&out)[4]) {
+    out[0] = __uint_as_float(raw.x); out[1] = __uint_as_float(raw.y);
+    out[2] = __uint_as_float(raw.z); out[3] = __uint_as_float(raw.w);
+}
+template <>
+__device__ __forceinline__ void unpack_vec<__nv_bfloat16>(const uint4& raw, float (&out)[8]) {
+    out[0] = bf16_lo(raw.x); out[1] = bf16_hi(raw.x); out[2] = bf16_lo(raw.y); out[3] = bf16_hi(raw.y);
+    out[4] = bf16_lo(raw.z); out[5] = bf16_hi(raw.z); out[6] = bf16_lo(raw.w); out[7] = bf16_hi(raw.w);
+}
+// floats that are exactly representable in T -> 16 bytes of T
+template <typename T>
+__device__ __forceinline__ uint4 pack_vec(const float (&x)[Vec16<T>::N]);
+template <>
+__device__ __forceinline__ uint4 pack_vec<float>(const float (&x)[4]) {
+    return make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
+}
+template <>
+__device__ __forceinline__ uint4 pack_vec<__nv_bfloat16>(const float (&x)[8]) {
+    // the values are bf16 already: their upper halves are the bit patterns
+    return make_uint4((__float_as_uint(x[0]) >> 16) | (__float_as_uint(x[1]) & 0xFFFF0000u),
+                      (__float_as_uint(x[2]) >> 16) | (__float_as_uint(x[3]) & 0xFFFF0000u),
+                      (__float_as_uint(x[4]) >> 16) | (__float_as_uint(x[5]) & 0xFFFF0000u),
+                      (__float_as_uint(x[6]) >> 16) | (__float_as_uint(x[7]) & 0xFFFF0000u));
+}
+// one element through a generic (e.g. shared-memory) pointer
+__device__ __forceinline__ float load_scalar_generic(const float* p) { return *p; }
+__device__ __forceinline__ float load_scalar_generic(const __nv_bfloat16* p) {
+    return __uint_as_float(((uint32_t)*reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+
 // ---- keyed permutation of [0,b) used to sample generators ---------------------
 // A 6-round balanced Feistel network on w bits (w even, 2^w >= b), cycle-walked
 // until the value falls below b.  Round keys come from splitmix64(seed).

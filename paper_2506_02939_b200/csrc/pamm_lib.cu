@@ -19,6 +19,7 @@
 #include "weight_grad_persist.cuh"
 #include "weight_grad_chunked.cuh"
 #include "linear_forward.cuh"
+#include "small_k.cuh"
 
 using namespace pamm;
 
@@ -188,6 +189,7 @@ constexpr int64_t FUSED_SCAN_LIMIT = 1ll << 24;
 // pass left behind) saves the histogram launch.
 pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const int32_t* products, const ContractWs& w,
                         cudaStream_t st) {
+    if (k <= SK_MAX_K) products = nullptr;     // the forward pass for so few generators leaves no counts
     const size_t hsmem = (size_t)k * 4;
     const int rpb = (int)w.rows_per_block;
     const int tbl_warps = scatter_table_warps(rpb, k);
@@ -293,6 +295,61 @@ pamm_status launch_weight_grad_simt(const void* C, int64_t ldc, int64_t k, int64
         launch(kern, grid, block, 0, st, true, (const T*)C, ldc, (int)k, n, Bt, ldb, m, (__nv_bfloat16*)dw.ptr, dw.ld, b_rows,
                dropped, accumulate ? 1 : 0);
     }
+    prof_end(PAMM_PROF_WEIGHT_GRAD, st);
+    return launch_status();
+}
+
+// ---- a handful of generators (k <= 8): three launches for the whole path ----
+template <typename T>
+pamm_status launch_small_forward(const void* X, int64_t ldx, int64_t b, int64_t n, int64_t k, uint64_t seed,
+                                 const int32_t* idx_in, int32_t* idx_out, void* C, int64_t ldc, float* c_invnorm,
+                                 void* f, int f_type, float* alpha, cudaStream_t st) {
+    constexpr int V = Vec16<T>::N;
+    const size_t smem = (size_t)k * round_up(n, V) * sizeof(T);
+    if (!ensure_dynamic_smem((const void*)compress_small_kernel<T>, smem)) return PAMM_ERR_CUDA;
+    // a row per warp while there are few rows; enough rows per CTA to pay for its copy of the generators otherwise
+    const int64_t rows_per_cta = std::max<int64_t>(SK_WARPS, (b + 4 * sm_count() - 1) / (4 * sm_count()));
+    const PermKey pk = make_perm_key(seed, (uint32_t)b);
+    prof_begin(PAMM_PROF_COMPRESS, st);
+    launch(compress_small_kernel<T>, dim3((unsigned)((b + rows_per_cta - 1) / rows_per_cta)), dim3(SK_THREADS), smem, st, true,
+           (const T*)X, ldx, b, n, (int)k, pk, idx_in, idx_out, (T*)C, ldc, c_invnorm, f, f_type, alpha, (int)rows_per_cta);
+    prof_end(PAMM_PROF_COMPRESS, st);
+    return launch_status();
+}
+
+template <typename T, typename OutT>
+void launch_wgrad_small(const void* C, int64_t ldc, int64_t k, int64_t n, const float* partials, int ranges, int64_t m_pad,
+                        int64_t m, float* Bt, int64_t ldb, const DwSpec& dw, bool accumulate, cudaStream_t st) {
+    const dim3 grid((unsigned)((m + SK_WG_COLS - 1) / SK_WG_COLS), (unsigned)((n + SK_WG_ROWS - 1) / SK_WG_ROWS));
+    if (dw.layout == PAMM_DW_MN)
+        launch(wgrad_small_kernel<T, OutT, true>, grid, dim3(SK_THREADS), 0, st, true, (const T*)C, ldc, (int)k, n, partials, ranges,
+               m_pad, m, Bt, ldb, (OutT*)dw.ptr, dw.ld, accumulate ? 1 : 0);
+    else
+        launch(wgrad_small_kernel<T, OutT, false>, grid, dim3(SK_THREADS), 0, st, true, (const T*)C, ldc, (int)k, n, partials, ranges,
+               m_pad, m, Bt, ldb, (OutT*)dw.ptr, dw.ld, accumulate ? 1 : 0);
+}
+
+template <typename T>
+pamm_status launch_small_backward(const void* C, int64_t ldc, int64_t n, const void* f, int f_type, const float* alpha,
+                                  const void* dY, int64_t ldy, int64_t b, int64_t m, int64_t k, float* Bt, int64_t ldb,
+                                  const DwSpec& dw, const ContractWs& w, cudaStream_t st) {
+    constexpr int V = Vec16<T>::N;
+    // one partial B~ (k rows) per row range, in the workspace's partial rows
+    int64_t ranges = std::max<int64_t>(1, std::min<int64_t>((b + 31) / 32, std::min<int64_t>(CT_MAX_CTAS / k, 2 * sm_count())));
+    const int64_t rows_per_range = (b + ranges - 1) / ranges;
+    ranges = (b + rows_per_range - 1) / rows_per_range;
+    const int64_t vecs = (m + V - 1) / V;
+    const int threads = (int)std::min<int64_t>(SK_CT_THREADS, round_up(vecs, 32));
+    const int64_t slabs = (vecs + threads - 1) / threads;
+    prof_begin(PAMM_PROF_CONTRACT, st);
+    launch(contract_small_kernel<T>, dim3((unsigned)ranges, (unsigned)slabs), dim3(threads), 0, st, true, f, f_type, alpha,
+           (const T*)dY, ldy, b, m, (int)k, (int)rows_per_range, w.partials, w.m_pad);
+    prof_end(PAMM_PROF_CONTRACT, st);
+    prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
+    if (dw.dt == PAMM_F32)
+        launch_wgrad_small<T, float>(C, ldc, k, n, w.partials, (int)ranges, w.m_pad, m, Bt, ldb, dw, false, st);
+    else
+        launch_wgrad_small<T, __nv_bfloat16>(C, ldc, k, n, w.partials, (int)ranges, w.m_pad, m, Bt, ldb, dw, false, st);
     prof_end(PAMM_PROF_WEIGHT_GRAD, st);
     return launch_status();
 }
@@ -550,6 +607,12 @@ pamm_status pamm_compress_fused(const void* X, int64_t ldx, int64_t b, int64_t n
     s = check_products_out(workspace, ws_bytes, b, k, 1);
     if (s != PAMM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
+    // a handful of generators: selection and compression in one launch, generator rows kept in shared memory
+    if (dt == PAMM_F32 && small_k_compress_supported<float>(n, k))
+        return launch_small_forward<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, f, (int)f_type, alpha, st);
+    if (dt == PAMM_BF16 && small_k_compress_supported<__nv_bfloat16>(n, k))
+        return launch_small_forward<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, f, (int)f_type,
+                                                   alpha, st);
     s = dt == PAMM_F32 ? launch_select<float>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st)
                        : launch_select<__nv_bfloat16>(X, ldx, b, n, k, seed, idx_in, idx_out, C, ldc, c_invnorm, st);
     if (s != PAMM_OK) return s;
@@ -664,6 +727,10 @@ pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, con
     s = check_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dw);
     if (s != PAMM_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
+    if (k <= SK_MAX_K)      // a handful of generators: no sort, two launches (the caller's B~, if any, is still filled)
+        return dt == PAMM_F32
+            ? launch_small_backward<float>(C, ldc, n, f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, dw, w, st)
+            : launch_small_backward<__nv_bfloat16>(C, ldc, n, f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, dw, w, st);
     const int32_t* pr = (const int32_t*)sort_products;
     s = dt == PAMM_F32 ? launch_contract<float>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st)
                        : launch_contract<__nv_bfloat16>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st);

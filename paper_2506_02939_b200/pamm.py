@@ -103,11 +103,21 @@ def _stream(stream) -> ctypes.c_void_p:
     return ctypes.c_void_p(s.cuda_stream)
 
 
+_prep_keep = None      # while a call is being prepared: the tensors it allocates, kept alive with the prepared call
+
+
+def _empty(*args, **kwargs) -> torch.Tensor:
+    t = torch.empty(*args, **kwargs)
+    if _prep_keep is not None:
+        _prep_keep.append(t)
+    return t
+
+
 def alloc_matrix(rows: int, cols: int, dtype, device="cuda") -> torch.Tensor:
     """rows x cols view whose row stride is padded so that every row starts 16-byte aligned."""
     per = 16 // torch.empty((), dtype=dtype).element_size()
     ld = (cols + per - 1) // per * per
-    return torch.empty((rows, ld), dtype=dtype, device=device)[:, :cols]
+    return _empty((rows, ld), dtype=dtype, device=device)[:, :cols]
 
 
 def workspace_bytes(kind: int, b: int, n: int, m: int, k: int, dtype: int) -> int:
@@ -118,20 +128,20 @@ def workspace_bytes(kind: int, b: int, n: int, m: int, k: int, dtype: int) -> in
 
 
 def alloc_workspace(kind: int, b: int, n: int, m: int, k: int, dtype: int, device="cuda") -> torch.Tensor:
-    return torch.empty(max(256, workspace_bytes(kind, b, n, m, k, dtype)), dtype=torch.uint8, device=device)
+    return _empty(max(256, workspace_bytes(kind, b, n, m, k, dtype)), dtype=torch.uint8, device=device)
 
 
 def draw_indices_host(b: int, k: int, seed: int) -> torch.Tensor:
-    out = torch.empty(k, dtype=torch.int32)
+    out = _empty(k, dtype=torch.int32)
     _check(_lib.pamm_draw_indices_host(b, k, seed, _ptr(out)), "pamm_draw_indices_host")
     return out
 
 
 def select_generators(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, c_invnorm=None, stream=None):
     b, n = X.shape
-    idx_out = torch.empty(k, dtype=torch.int32, device=X.device) if idx_out is None else idx_out
+    idx_out = _empty(k, dtype=torch.int32, device=X.device) if idx_out is None else idx_out
     C = alloc_matrix(k, n, X.dtype, X.device) if C is None else C
-    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=X.device) if c_invnorm is None else c_invnorm
+    c_invnorm = _empty(2 * k, dtype=torch.float32, device=X.device) if c_invnorm is None else c_invnorm
     _check(_lib.pamm_select_generators(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out),
                                        _ptr(C), _ld(C), _ptr(c_invnorm), _stream(stream)), "pamm_select_generators")
     return idx_out, C, c_invnorm
@@ -149,7 +159,7 @@ def _ft(f: torch.Tensor) -> int:
 
 
 def _new_f(shape, f_dtype, device):
-    return torch.empty(shape, dtype=torch.int32 if f_dtype is None else f_dtype, device=device)
+    return _empty(shape, dtype=torch.int32 if f_dtype is None else f_dtype, device=device)
 
 
 def _bytes(t) -> int:
@@ -162,7 +172,7 @@ def compress(X, C, c_invnorm, f=None, alpha=None, sort_products=None, f_dtype=No
     b, n = X.shape
     k = C.shape[0]
     f = _new_f(b, f_dtype, X.device) if f is None else f
-    alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
+    alpha = _empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
     _check(_lib.pamm_compress(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), _ptr(f), _ft(f),
                               _ptr(alpha), _ptr(sort_products), _bytes(sort_products), _stream(stream)), "pamm_compress")
     return f, alpha
@@ -174,7 +184,7 @@ def compress_projections(X, C, c_invnorm, sets: int, f=None, alpha=None, sort_pr
     b, n = X.shape
     k = C.shape[0] // sets
     f = _new_f((sets, b), f_dtype, X.device) if f is None else f
-    alpha = torch.empty((sets, b), dtype=torch.float32, device=X.device) if alpha is None else alpha
+    alpha = _empty((sets, b), dtype=torch.float32, device=X.device) if alpha is None else alpha
     _check(_lib.pamm_compress_projections(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, sets, _ptr(c_invnorm), _ptr(f),
                                           _ft(f), _ptr(alpha), f.stride(0), _ptr(sort_products), _bytes(sort_products),
                                           _stream(stream)), "pamm_compress_projections")
@@ -188,8 +198,8 @@ def compress_eps(X, C, c_invnorm, eps: float, f=None, alpha=None, dropped=None, 
     b, n = X.shape
     k = C.shape[0]
     f = _new_f(b, f_dtype, X.device) if f is None else f
-    alpha = torch.empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
-    dropped = torch.empty(1, dtype=torch.int32, device=X.device) if dropped is None else dropped
+    alpha = _empty(b, dtype=torch.float32, device=X.device) if alpha is None else alpha
+    dropped = _empty(1, dtype=torch.int32, device=X.device) if dropped is None else dropped
     _check(_lib.pamm_compress_eps(_ptr(X), _ld(X), b, n, _dt(X), _ptr(C), _ld(C), k, _ptr(c_invnorm), float(eps), _ptr(f),
                                   _ft(f), _ptr(alpha), _ptr(dropped), _ptr(sort_products), _bytes(sort_products),
                                   _stream(stream)), "pamm_compress_eps")
@@ -236,11 +246,11 @@ def compress_fused(X, k: int, seed: int = 0, idx_in=None, idx_out=None, C=None, 
                    sort_products=None, f_dtype=None, stream=None):
     b, n = X.shape
     dev = X.device
-    idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
+    idx_out = _empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
     C = alloc_matrix(k, n, X.dtype, dev) if C is None else C
-    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
+    c_invnorm = _empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
     f = _new_f(b, f_dtype, dev) if f is None else f
-    alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
+    alpha = _empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
     _check(_lib.pamm_compress_fused(_ptr(X), _ld(X), b, n, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out), _ptr(C),
                                     _ld(C), _ptr(c_invnorm), _ptr(f), _ft(f), _ptr(alpha), _ptr(sort_products),
                                     _bytes(sort_products), _stream(stream)), "pamm_compress_fused")
@@ -254,11 +264,11 @@ def linear_forward(X, W, k: int, seed: int = 0, idx_in=None, Z=None, idx_out=Non
     m = W.shape[1]
     dev = X.device
     Z = alloc_matrix(b, m, X.dtype, dev) if Z is None else Z
-    idx_out = torch.empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
+    idx_out = _empty(k, dtype=torch.int32, device=dev) if idx_out is None else idx_out
     C = alloc_matrix(k, n, X.dtype, dev) if C is None else C
-    c_invnorm = torch.empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
+    c_invnorm = _empty(2 * k, dtype=torch.float32, device=dev) if c_invnorm is None else c_invnorm
     f = _new_f(b, f_dtype, dev) if f is None else f
-    alpha = torch.empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
+    alpha = _empty(b, dtype=torch.float32, device=dev) if alpha is None else alpha
     _check(_lib.pamm_linear_forward(_ptr(X), _ld(X), b, n, _ptr(W), _ld(W), m, _dt(X), k, seed, _ptr(idx_in), _ptr(idx_out),
                                     _ptr(C), _ld(C), _ptr(c_invnorm), _ptr(Z), _ld(Z), _ptr(f), _ft(f), _ptr(alpha),
                                     _ptr(sort_products), _bytes(sort_products), _stream(stream)), "pamm_linear_forward")
@@ -315,6 +325,45 @@ def qkv_step_host(X_host, dY_host, k: int, seed: int, dW_host, arena, f_host=Non
                                    _ptr(f_host), _ptr(alpha_host), _ptr(arena), arena.numel(), _stream(stream)),
            "pamm_qkv_step_host")
     return dW_host
+
+
+class _RecordingLib:
+    """Stands in for the library while a call is being prepared: notes the C function and its marshalled arguments."""
+
+    def __init__(self, real):
+        self._real, self.calls = real, []
+
+    def __getattr__(self, name):
+        fn = getattr(self._real, name)
+
+        def note(*cargs):
+            self.calls.append((name, fn, cargs))
+            return OK
+        return note
+
+
+def prepared(call, *args, **kwargs):
+    """Marshal once, call often.  ``prepared(pamm.compress_fused, X, k, seed, idx_out=..., ...)`` runs nothing; it returns a
+    zero-argument callable that repeats exactly that C call (same pointers, sizes, seed and stream), skipping the
+    Python-side marshalling -- for loops where a step is only a few microseconds of GPU work.  Outputs the call
+    allocates itself stay alive with the callable but are not handed out: pass in the ones you want to read."""
+    global _lib, _prep_keep
+    real, rec = _lib, _RecordingLib(_lib)
+    _lib, _prep_keep = rec, []
+    try:
+        call(*args, **kwargs)
+        keep = (args, kwargs, _prep_keep)          # the tensors behind the pointers, the call's own allocations included
+    finally:
+        _lib, _prep_keep = real, None
+    if len(rec.calls) != 1:
+        raise ValueError("prepared() takes a binding function that makes exactly one library call")
+    name, fn, cargs = rec.calls[0]
+
+    def run(_fn=fn, _cargs=cargs, _name=name, _keep=keep):
+        code = _fn(*_cargs)
+        if code != OK:
+            raise PammError(code, _name)
+    return run
 
 
 def selftest_bounded_wait(stream=None) -> None:

@@ -5,7 +5,7 @@ What is compared, and how tightly:
 * f: bit-exact, except rows whose two best scores differ by less than 1e-6 relative in the
   oracle (counted as ``near_tie``).  A mismatch with a larger gap is tolerated only when the
   two competing scores are closer than the rounding of their fp32 n-term sums can resolve,
-  ``4 sqrt(n) 2^-24 sum_l |X_il C_jl| / ||C_j||`` for each competitor (counted as
+  ``2 sqrt(n) 2^-24 sum_l |X_il C_jl| / ||C_j||`` for each competitor (counted as
   ``explained_by_rounding``, at most max(2, b/2000) rows); anything else fails.
 * alpha, B~, dW~: the relative Frobenius error the method is specified with (1e-5 for fp32
   inputs, 1e-2 for bf16 inputs with fp32 accumulation), a second Frobenius line at what fp32

@@ -157,3 +157,28 @@ def test_draw_indices_non_power_of_two_uniform():
     expect = seeds * k / b
     chi2 = float(((counts - expect) ** 2 / expect).sum())
     assert chi2 < 36 + 5 * np.sqrt(72), chi2
+
+
+def test_prepared_calls_repeat_one_library_call():
+    out = torch.zeros(8, dtype=torch.int32)
+
+    def draw(seed):
+        pamm._check(pamm._lib.pamm_draw_indices_host(1000, 8, seed, pamm._ptr(out)), "pamm_draw_indices_host")
+
+    run = pamm.prepared(draw, 11)
+    assert torch.all(out == 0)                                  # preparing runs nothing
+    run()
+    assert torch.equal(out, pamm.draw_indices_host(1000, 8, 11))
+    out.zero_()
+    run()
+    assert torch.equal(out, pamm.draw_indices_host(1000, 8, 11))
+    # the call's own allocations stay alive with the callable
+    keep_alive = pamm.prepared(pamm.draw_indices_host, 1000, 8, 3)
+    keep_alive()
+    with pytest.raises(ValueError):
+        pamm.prepared(lambda: None)
+    bad = pamm.prepared(draw, 11)
+    assert pamm._lib is not None and callable(bad)
+    failing = pamm.prepared(lambda: pamm._check(pamm._lib.pamm_draw_indices_host(4, 8, 0, pamm._ptr(out)), "draw"))
+    with pytest.raises(pamm.PammError):
+        failing()                                               # k > b is reported when the call is made

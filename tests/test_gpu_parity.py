@@ -186,6 +186,37 @@ def test_device_side_problems_raise_a_status_not_a_fault():
     assert torch.all(Bt[1:] == 0)
 
 
+def test_few_generators_take_the_three_launch_path():
+    # k <= 8: selection + compression in one launch, contraction without a sort, reduction + product in one launch
+    X, dY = synth.random_case(3000, 200, 392, "bf16", seed=19, centres=6, dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    n0 = pamm.launch_count()
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, 6, 3)
+    Bt = pamm.alloc_matrix(6, 392, torch.float32)
+    dW = pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt)
+    assert pamm.launch_count() - n0 == 3
+    # the same selection and the same assignment as the general kernels give
+    idx2, C2, invn2 = pamm.select_generators(Xd, 6, 3)
+    f2, alpha2 = pamm.compress(Xd, C2, invn2)
+    assert torch.equal(idx, idx2) and torch.equal(C.view(torch.int16), C2.view(torch.int16))
+    assert torch.allclose(invn, invn2, rtol=1e-6, atol=0) and torch.equal(f, f2)
+    assert torch.allclose(alpha, alpha2, rtol=1e-5, atol=1e-7)
+    # caller's indices that are out of range or repeated: clamped, kept, reported -- as the selection kernel does
+    bad = torch.tensor([3, 99999, 7, 7], dtype=torch.int32, device="cuda")
+    idx, *_ = pamm.compress_fused(Xd, 4, idx_in=bad)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
+    assert idx.cpu().tolist() == [3, 2999, 7, 7]
+    # an assignment outside [0, k) is skipped and reported by the sort-free contraction too
+    f[10] = 6
+    Bt_bad = pamm.alloc_matrix(6, 392, torch.float32)
+    pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt_bad)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
+    keep = np.ones(3000, bool)
+    keep[10] = False
+    ref = orc.contract(np.where(keep, f.cpu().numpy(), 0).astype(np.int32), np.where(keep, alpha.cpu().numpy(), 0.0), dY, 6)
+    assert parity.rel_fro(Bt_bad.cpu().numpy(), ref) <= 1e-5
+
+
 def test_unfused_stage_inputs_from_elsewhere():
     # contract / weight_grad accept any (f, alpha, B~), not only what compress produced
     rng = np.random.default_rng(12)
@@ -338,7 +369,7 @@ def test_narrow_assignment_storage(f_dtype, b, n, m, k, dtype):
 
 # ---- the counts of f that the forward pass leaves for the backward pass ----
 
-@pytest.mark.parametrize("b,n,m,k,dtype", [(5000, 136, 264, 40, "bf16"), (3000, 64, 72, 900, "bf16"), (2048, 72, 96, 4, "f32")])
+@pytest.mark.parametrize("b,n,m,k,dtype", [(5000, 136, 264, 40, "bf16"), (3000, 64, 72, 900, "bf16"), (2048, 72, 96, 12, "f32")])
 def test_sort_products_of_the_forward_pass(b, n, m, k, dtype):
     # tensor-core compress, the three-launch sort (many generators), CUDA-core compress
     X, dY = synth.random_case(b, n, m, dtype, seed=61, centres=max(2, k // 3), dy_scale=1e-3)
