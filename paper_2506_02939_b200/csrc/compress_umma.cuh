@@ -209,51 +209,70 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
             ptx::prefetch_tensormap(&tm_x);
             ptx::prefetch_tensormap(&tm_c);
             const uint64_t stream_policy = ptx::l2_policy_evict_first();   // X is read once; C stays in L2
-            // pipeline step `it` = (row super tile, pass = (group, chunk), 64-column step), flattened
-            const uint32_t per_super = (uint32_t)(passes * ksteps);
-            const uint32_t total = (uint32_t)((r1 - r0 + super_rows - 1) / super_rows) * per_super;
-            auto issue = [&](uint32_t at, bool with_x, bool with_c, bool arm) {
-                const int64_t st = r0 + (int64_t)(at / per_super) * super_rows;
-                const int pass = (int)((at % per_super) / (uint32_t)ksteps), ks = (int)(at % (uint32_t)ksteps);
-                const int g = pass / num_chunks, ch = pass % num_chunks;
-                const int s = at % stages;
-                uint8_t* stage = tiles + (size_t)s * stage_bytes;
-                uint32_t bytes = (uint32_t)n_chunk * 128u;
+            // pipeline step = (row super tile, pass = (group, chunk), 64-column step).  The cursor walks the steps with
+            // additions only: what happens between a stage falling free and its copies being issued is on the critical
+            // path of a pipeline that is bound by the bytes it keeps in flight
+            struct Cursor {
+                int64_t st;          // first row of the super tile
+                int g, ch, ks, s;    // group, chunk, column step, ring stage
+                uint32_t phase;      // parity of the stage's use
                 int boxes[MT];
+                uint32_t x_bytes;
+            };
+            auto set_tile = [&](Cursor& c) {
+                c.x_bytes = 0;
 #pragma unroll
                 for (int mt = 0; mt < MT; ++mt) {
-                    const int64_t rows = min((int64_t)CU_TILE_M, r1 - (st + (int64_t)mt * CU_TILE_M));
-                    boxes[mt] = rows > 0 ? (int)((rows + CU_BOX_ROWS - 1) / CU_BOX_ROWS) : 0;
-                    bytes += (uint32_t)boxes[mt] * (CU_BOX_ROWS * 128u);
+                    const int64_t rows = min((int64_t)CU_TILE_M, r1 - (c.st + (int64_t)mt * CU_TILE_M));
+                    c.boxes[mt] = rows > 0 ? (int)((rows + CU_BOX_ROWS - 1) / CU_BOX_ROWS) : 0;
+                    c.x_bytes += (uint32_t)c.boxes[mt] * (CU_BOX_ROWS * 128u);
                 }
-                if (arm) ptx::mbar_arrive_expect_tx(&s_full[s], bytes);
+            };
+            auto advance = [&](Cursor& c) {
+                if (++c.s == stages) { c.s = 0; c.phase ^= 1u; }
+                if (++c.ks < ksteps) return;
+                c.ks = 0;
+                if (++c.ch == num_chunks) { c.ch = 0; ++c.g; }
+                if (c.g < groups) return;
+                c.g = 0;
+                c.st += super_rows;
+                set_tile(c);
+            };
+            auto issue = [&](const Cursor& c, bool with_x, bool with_c, bool arm) {
+                uint8_t* stage = tiles + (size_t)c.s * stage_bytes;
+                if (arm) ptx::mbar_arrive_expect_tx(&s_full[c.s], c.x_bytes + (uint32_t)n_chunk * 128u);
                 if (with_x) {
                     // the tile comes back once per pass: only its last visit may push it out of L2 early
-                    const bool last_pass = pass + 1 == passes;
+                    const bool last_pass = c.g + 1 == groups && c.ch + 1 == num_chunks;
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
-                        for (int q = 0; q < boxes[mt]; ++q) {
+                        for (int q = 0; q < c.boxes[mt]; ++q) {
                             uint8_t* dst = stage + mt * CU_X_TILE_BYTES + q * (CU_BOX_ROWS * 128);
-                            const int32_t y = (int32_t)(st + mt * CU_TILE_M + q * CU_BOX_ROWS);
-                            if (last_pass) ptx::tma_load_2d_hint(dst, &tm_x, ks * CU_BLOCK_K, y, &s_full[s], stream_policy);
-                            else           ptx::tma_load_2d(dst, &tm_x, ks * CU_BLOCK_K, y, &s_full[s]);
+                            const int32_t y = (int32_t)(c.st + mt * CU_TILE_M + q * CU_BOX_ROWS);
+                            if (last_pass) ptx::tma_load_2d_hint(dst, &tm_x, c.ks * CU_BLOCK_K, y, &s_full[c.s], stream_policy);
+                            else           ptx::tma_load_2d(dst, &tm_x, c.ks * CU_BLOCK_K, y, &s_full[c.s]);
                         }
                 }
                 if (with_c)
-                    ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, ks * CU_BLOCK_K, g * k + ch * n_chunk, &s_full[s]);
+                    ptx::tma_load_2d(stage + MT * CU_X_TILE_BYTES, &tm_c, c.ks * CU_BLOCK_K, c.g * k + c.ch * n_chunk, &s_full[c.s]);
             };
+            const uint32_t total = (uint32_t)((r1 - r0 + super_rows - 1) / super_rows) * (uint32_t)(passes * ksteps);
+            Cursor cur;
+            cur.st = r0; cur.g = 0; cur.ch = 0; cur.ks = 0; cur.s = 0; cur.phase = 0;
+            set_tile(cur);
             uint32_t it = 0;
             bool ok = true;
             if (x_is_ready) {     // fill the ring with X, then wait for the kernel before, then add the C tiles
                 const uint32_t ahead = total < (uint32_t)stages ? total : (uint32_t)stages;
-                for (uint32_t a = 0; a < ahead; ++a) issue(a, true, false, true);
+                Cursor pre = cur;
+                for (uint32_t a = 0; a < ahead; ++a, advance(pre)) issue(pre, true, false, true);
                 grid_dependency_wait();
-                for (uint32_t a = 0; a < ahead; ++a) issue(a, false, true, false);
+                for (uint32_t a = 0; a < ahead; ++a, advance(cur)) issue(cur, false, true, false);
                 it = ahead;
             }
-            for (; it < total; ++it) {
-                if (!ptx::mbar_wait(&s_empty[it % stages], ((it / stages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                issue(it, true, true, true);
+            for (; it < total; ++it, advance(cur)) {
+                if (!ptx::mbar_wait(&s_empty[cur.s], cur.phase ^ 1u, abort_flag)) { ok = false; break; }
+                issue(cur, true, true, true);
             }
             if (!ok) {
                 raise_status(DEV_TIMEOUT);
@@ -271,7 +290,8 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
         // ---------------- MMA issuer ----------------
         if (ptx::elect_one()) {
             const uint32_t idesc = ptx::umma_idesc_bf16(CU_TILE_M, (uint32_t)n_chunk);
-            uint32_t it = 0, unit = 0;
+            uint32_t unit = 0, sph = 0;
+            int s = 0;               // ring stage and the parity of its use, advanced without divisions
             bool ok = true;
             for (int64_t st = r0; st < r1 && ok; st += super_rows) {
                 for (int pass = 0; pass < passes && ok; ++pass, ++unit) {
@@ -279,9 +299,8 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                     if (!ptx::mbar_wait(&s_tempty[buf], uph ^ 1u, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     const uint32_t d_base = tmem_base + buf * (uint32_t)(MT * n_chunk);
-                    for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                        const int s = it % stages;
-                        if (!ptx::mbar_wait(&s_full[s], (it / stages) & 1u, abort_flag)) { ok = false; break; }
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        if (!ptx::mbar_wait(&s_full[s], sph, abort_flag)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
                         const uint32_t stage_addr = ptx::smem_u32(tiles + (size_t)s * stage_bytes);
                         const uint64_t desc_b = ptx::umma_desc_k_sw128(stage_addr + MT * CU_X_TILE_BYTES);
@@ -295,6 +314,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                                                (ks | kk) != 0);
                         }
                         ptx::umma_commit(&s_empty[s]);   // frees the stage once these MMAs have read it
+                        if (++s == stages) { s = 0; sph ^= 1u; }
                     }
                     if (ok) ptx::umma_commit(&s_tfull[buf]);
                 }

@@ -139,7 +139,8 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
             // X and W were complete before the kernel in front of this one (the generator selection)
             // started; C comes from it and is waited for where the first score item begins
             bool c_ready = false;
-            uint32_t it = 0;
+            uint32_t it = 0, sph = 0;
+            int s = 0;               // ring stage and the parity of its use
             bool ok = true;
             for (int64_t t = blockIdx.x; t < items && ok; t += gridDim.x) {
                 int64_t rb, ct;
@@ -149,8 +150,7 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 const int units = score ? num_chunks : 1;
                 for (int u = 0; u < units && ok; ++u) {
                     for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                        const int s = it % stages;
-                        if (!ptx::mbar_wait(&s_empty[s], ((it / stages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!ptx::mbar_wait(&s_empty[s], sph ^ 1u, abort_flag)) { ok = false; break; }
                         uint8_t* stage = tiles + (size_t)s * LF_STAGE_BYTES;
                         const uint32_t b_bytes = score ? (uint32_t)n_chunk * 128u : (uint32_t)LF_B_BYTES;
                         ptx::mbar_arrive_expect_tx(&s_full[s], LF_A_BYTES + b_bytes);
@@ -163,6 +163,7 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                                 ptx::tma_load_2d(stage + LF_A_BYTES + q * 8192, &tm_w, (int32_t)(ct * LF_TILE_N + q * 64),
                                                  ks * LF_BLOCK_K, &s_full[s]);
                         }
+                        if (++s == stages) { s = 0; sph ^= 1u; }
                     }
                 }
             }
@@ -182,7 +183,8 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
         if (ptx::elect_one()) {
             const uint32_t idesc_z = ptx::umma_idesc_bf16(LF_TILE_M, LF_TILE_N) | (1u << 16);     // B (W) is MN-major
             const uint32_t idesc_s = ptx::umma_idesc_bf16(LF_TILE_M, (uint32_t)n_chunk);          // B (C) is K-major
-            uint32_t it = 0, unit = 0;
+            uint32_t unit = 0, sph = 0;
+            int s = 0;               // ring stage and the parity of its use
             bool ok = true;
             for (int64_t t = blockIdx.x; t < items && ok; t += gridDim.x) {
                 int64_t rb, ct;
@@ -194,9 +196,8 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     if (!ptx::mbar_wait(&s_tempty[buf], uph ^ 1u, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
                     const uint32_t d_addr = tmem_base + buf * (uint32_t)LF_TILE_N;
-                    for (int ks = 0; ks < ksteps; ++ks, ++it) {
-                        const int s = it % stages;
-                        if (!ptx::mbar_wait(&s_full[s], (it / stages) & 1u, abort_flag)) { ok = false; break; }
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        if (!ptx::mbar_wait(&s_full[s], sph, abort_flag)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
                         const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)s * LF_STAGE_BYTES);
                         const uint32_t b_addr = a_addr + LF_A_BYTES;
@@ -213,6 +214,7 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                                                idesc_z, (ks | kk) != 0);
                         }
                         ptx::umma_commit(&s_empty[s]);
+                        if (++s == stages) { s = 0; sph ^= 1u; }
                     }
                     if (ok) ptx::umma_commit(&s_tfull[buf]);
                 }

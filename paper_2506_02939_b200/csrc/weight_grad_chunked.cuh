@@ -155,7 +155,7 @@ weight_grad_chunked_kernel(const __grid_constant__ CUtensorMap tm_c, const __gri
             ptx::tc_fence_after_sync();
 #pragma unroll
             for (int h = 0; h < 2; ++h)
-                wg_epilogue_half<OutT, 1>(&tm_w, tmem_base + (uint32_t)(s * WG_TILE), &s_tempty[s],
+                wg_epilogue_half<OutT>(&tm_w, tmem_base + (uint32_t)(s * WG_TILE), &s_tempty[s],
                                        sOut + h * WgOut<OutT>::HALF_BYTES, quad, lane, h, leader, swap ? n0 : m0,
                                        swap ? m0 : n0, beta, accumulate != 0, ok);
         }

@@ -16,8 +16,7 @@
 namespace pamm {
 
 constexpr int WG_TILE = 128;                 // output tile: 128 x 128
-constexpr int WG_EPI_WARPS = 8;              // quadrant (TMEM lanes) x column half
-constexpr int WG_EPI_GROUP_THREADS = 128;    // the four warps that share a column half
+constexpr int WG_EPI_GROUP_THREADS = 128;    // the four epilogue warps
 constexpr uint32_t WG_EPI_BARRIER0 = 1;      // named barriers 1 and 2: one per column half
 
 // Shared-memory operand descriptor, MN-major, 128-byte swizzle: blocks of 64
@@ -68,40 +67,6 @@ __device__ __forceinline__ void load_bt8(const float* __restrict__ Bt, int64_t l
     }
 }
 
-// Converts the 128-column block of B~ that starts at column m0 (kc generator rows, zero rows
-// past k) into the bf16 hi / lo operand blocks, with `nth` threads of which the caller is
-// number `t` (whole warps, t - lane a multiple of 32).  Items (one generator x 8 columns)
-// are dealt round-robin, so a warp's 32 items always lie in one group of 16 generators;
-// BATCH rounds of loads are in flight together, and after every round each warp announces
-// its share on the group's barrier (eight warp-arrivals complete a group).
-template <int BATCH>
-__device__ __forceinline__ void convert_bt_block(const float* __restrict__ Bt, int64_t ldb, int k, int64_t m, int kc,
-                                                 int64_t m0, uint8_t* sBhi, uint8_t* sBlo, uint32_t blk_bytes,
-                                                 uint64_t* s_bfull, int t, int nth) {
-    const int items = kc * 16;
-    const bool full_cols = m0 + WG_TILE <= m;
-    const int lane = threadIdx.x & 31;
-    for (int base = 0; base < items; base += BATCH * nth) {
-        float4 a4[BATCH], b4[BATCH];
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) {     // every load of the batch first
-            const int idx = base + u * nth + t;
-            a4[u] = b4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (idx < items && (idx >> 4) < k) load_bt8(Bt, ldb, idx >> 4, m0 + (idx & 15) * 8, m, full_cols, a4[u], b4[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) {
-            const int idx = base + u * nth + t;
-            if (idx - lane < items) {         // warp-uniform: items is a multiple of 256
-                split_store_hi_lo(sBhi, sBlo, blk_bytes, idx >> 4, idx & 15, a4[u], b4[u]);
-                ptx::fence_proxy_async();     // generic-proxy stores -> visible to the tensor core's async proxy
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&s_bfull[idx >> 8]);
-            }
-        }
-    }
-}
-
 // Staging of the output tile in shared memory: TMA boxes of 128 rows x 128 bytes
 // (32 fp32 or 64 bf16 columns) in the 128-byte swizzle.  A column half of the tile
 // (64 columns) is two fp32 boxes or one bf16 box.
@@ -115,16 +80,16 @@ template <> struct WgOut<__nv_bfloat16> {
     static constexpr int HALF_BYTES = WG_TILE * 128;
 };
 
-// Epilogue of one output tile for one warp: the warp owns TMEM lanes [32 quad, 32 quad + 32)
-// (= 32 rows of the tile) and the 64 columns of column half `h`.  Accumulators go
+// Epilogue of one column half of an output tile for one warp: the warp owns TMEM lanes
+// [32 quad, 32 quad + 32) (= 32 rows of the tile) and handles the 64 columns of half `h`.  Accumulators go
 // TMEM -> registers (scaled by beta) -> the half's staging area; the four warps of the half
 // then meet and one thread hands the area to the TMA engine (store, or reduce-add for
 // gradient accumulation).  `x0`, `y0` are the tile's column / row in the output matrix.
 // The accumulator is handed back (`tempty`) as soon as it sits in registers.
-// `ok == false` keeps only the barrier sequence going.  PENDING = how many of the leader's
-// earlier stores may still be reading shared memory when this one stages its data: 0 when the
-// leader serves this half only, 1 when it alternates between the two halves' staging areas.
-template <typename OutT, int PENDING>
+// `ok == false` keeps only the barrier sequence going.  The two halves have a staging area
+// each and alternate, so the store of one half is still reading shared memory while the other
+// is staged: the leader waits until at most one of its earlier stores is still reading.
+template <typename OutT>
 __device__ __forceinline__ void wg_epilogue_half(const CUtensorMap* tm_w, uint32_t tmem_acc, uint64_t* tempty,
                                                  uint8_t* half_stage, int quad, int lane, int h, bool leader, int x0, int y0,
                                                  float beta, bool accumulate, bool ok) {
@@ -147,7 +112,7 @@ __device__ __forceinline__ void wg_epilogue_half(const CUtensorMap* tm_w, uint32
         }
     }
     // the store that last used this staging area must have read it before it is overwritten
-    if (leader) ptx::bulk_wait_group_read<PENDING>();
+    if (leader) ptx::bulk_wait_group_read<1>();
     ptx::named_barrier(WG_EPI_BARRIER0 + (uint32_t)h, WG_EPI_GROUP_THREADS);
     if (ok) {
         if constexpr (sizeof(OutT) == 4) {
