@@ -241,6 +241,10 @@ contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, 
     const int me = blockIdx.x;
     grid_dependency_wait();     // f and the histograms come from kernels before
     grid_launch_dependents();
+    const int64_t i0 = (int64_t)me * rows_per_block;
+    const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
+    // the keys of the first chunk travel while the column sums are formed
+    int32_t first_key = i0 + tid < i1 ? load_index(f, f_type, i0 + tid) : -1;
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < k; j0 += SORT_BLK) {
@@ -311,13 +315,11 @@ contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, 
     }
     if (me == 0 && tid == 0) seg_start[k] = s_carry;
 
-    const int64_t i0 = (int64_t)me * rows_per_block;
-    const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
     for (int64_t c0 = i0; c0 < i1; c0 += SORT_BLK) {
         const int64_t i = c0 + tid;
         int32_t key = -1;
         if (i < i1) {
-            key = load_index(f, f_type, i);
+            key = c0 == i0 ? first_key : load_index(f, f_type, i);
             if (key < 0 || key >= k) key = -1;
         }
         scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), k, s_next, s_tbl, perm, b);
