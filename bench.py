@@ -293,10 +293,24 @@ def run_cuda(args):
     K = args.steps
     KINDS = (pamm.PROF_COMPRESS, pamm.PROF_CONTRACT, pamm.PROF_WEIGHT_GRAD)
 
+    # Steps of the timed region that carry events: one in PROF_EVERY for the kernels and as many for
+    # the stages; a run too short for that carries one kernel step, its last, and no stage step.
+    if K >= 4 * PROF_EVERY:
+        kernel_at = set(range(0, K, PROF_EVERY))
+        stage_at = set(range(PROF_EVERY // 2, K, PROF_EVERY))
+    else:
+        kernel_at, stage_at = {K - 1}, set()
+    event_pool = []
+
     def new_event():
+        if event_pool:
+            return event_pool.pop()
         e = torch.cuda.Event(enable_timing=True)
         e.record(stream)          # creates the underlying CUDA event, whose handle the library records later
         return e
+
+    # the events the timed region will use exist before it starts
+    event_pool.extend([new_event() for _ in range(2 * len(KINDS) * len(kernel_at))])
 
     def kernel_step(seed):
         """One step with an event pair around each step's main kernel."""
@@ -329,9 +343,9 @@ def run_cuda(args):
     sampler.start()
     t_begin.record(stream)
     for s in range(K):
-        if s % PROF_EVERY == 0 and K >= PROF_EVERY:
+        if s in kernel_at:
             kernel_samples.append(kernel_step(w.index_seed + s))
-        elif s % PROF_EVERY == PROF_EVERY // 2 and K >= PROF_EVERY:
+        elif s in stage_at:
             stage_samples.append(staged_step(w.index_seed + s))
         else:
             step(w.index_seed + s)
