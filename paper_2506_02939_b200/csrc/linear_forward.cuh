@@ -71,11 +71,12 @@ inline LinearForwardPlan linear_forward_plan(int64_t b, int64_t m, int64_t k, in
 
 // Item t -> (row block, column tile); `per_block` items per row block: the column tiles of W and,
 // if there is one, the score item (column tile == col_tiles).
-__device__ __forceinline__ void lf_decode(int64_t t, int64_t row_blocks, int64_t per_block, int64_t& rb, int64_t& ct) {
-    const int64_t per_group = (int64_t)LF_GROUP * per_block;
+__device__ __forceinline__ void lf_decode(int64_t t, int64_t row_blocks, int64_t per_block, int64_t& rb, int64_t& ct,
+                                          int group = LF_GROUP) {
+    const int64_t per_group = (int64_t)group * per_block;
     const int64_t grp = t / per_group;
-    const int64_t first = grp * LF_GROUP;
-    const int64_t in_group = min((int64_t)LF_GROUP, row_blocks - first);     // the last group may be short
+    const int64_t first = grp * group;
+    const int64_t in_group = min((int64_t)group, row_blocks - first);     // the last group may be short
     const int64_t r = t - grp * per_group;
     ct = r / in_group;
     rb = first + r % in_group;
@@ -88,6 +89,87 @@ struct LinearForwardOut {
     int rows_per_block;      // that partition
     int f_type;
 };
+
+// Epilogue of a 128 x 256 tile of Z for one thread (one row): TMEM -> registers -> bf16 -> swizzled
+// staging area -> TMA store, 64 columns at a time.  `release()` hands the accumulator back once its
+// last columns are in registers (called by every thread of the warp, converged).
+template <typename Release>
+__device__ __forceinline__ void lf_store_z_tile(uint32_t t_base, uint8_t* slab, int row_in_tile, bool leader,
+                                                const CUtensorMap* tm_z, int32_t col0, int32_t row0, Release release) {
+#pragma unroll 1
+    for (int sl = 0; sl < LF_TILE_N / 64; ++sl) {
+        uint32_t v0[32], v1[32];
+        ptx::tmem_ld_32x32(t_base + (uint32_t)(sl * 64), v0);
+        ptx::tmem_ld_32x32(t_base + (uint32_t)(sl * 64 + 32), v1);
+        ptx::tmem_ld_wait();
+        if (sl == LF_TILE_N / 64 - 1) {          // the accumulator is in registers: hand it back
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            release();
+        }
+        if (leader) ptx::bulk_wait_group_read<0>();     // the previous store has read the staging area
+        ptx::named_barrier(1, 128);
+        uint8_t* d0 = slab + row_in_tile * 128;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            *reinterpret_cast<uint4*>(d0 + ((c ^ (row_in_tile & 7)) << 4)) =
+                make_uint4(pack_bf16(__uint_as_float(v0[8 * c]), __uint_as_float(v0[8 * c + 1])),
+                           pack_bf16(__uint_as_float(v0[8 * c + 2]), __uint_as_float(v0[8 * c + 3])),
+                           pack_bf16(__uint_as_float(v0[8 * c + 4]), __uint_as_float(v0[8 * c + 5])),
+                           pack_bf16(__uint_as_float(v0[8 * c + 6]), __uint_as_float(v0[8 * c + 7])));
+            *reinterpret_cast<uint4*>(d0 + (((c + 4) ^ (row_in_tile & 7)) << 4)) =
+                make_uint4(pack_bf16(__uint_as_float(v1[8 * c]), __uint_as_float(v1[8 * c + 1])),
+                           pack_bf16(__uint_as_float(v1[8 * c + 2]), __uint_as_float(v1[8 * c + 3])),
+                           pack_bf16(__uint_as_float(v1[8 * c + 4]), __uint_as_float(v1[8 * c + 5])),
+                           pack_bf16(__uint_as_float(v1[8 * c + 6]), __uint_as_float(v1[8 * c + 7])));
+        }
+        ptx::fence_proxy_async();
+        ptx::named_barrier(1, 128);
+        if (leader) {
+            ptx::tma_store_2d(tm_z, slab, col0 + sl * 64, row0);
+            ptx::bulk_commit_group();
+        }
+    }
+}
+
+// One chunk of generators for one row: the running (best score, dot product, argmax) over the
+// chunk's n_chunk accumulator columns, the next 16 columns in flight while 16 are compared.
+__device__ __forceinline__ void lf_score_chunk(uint32_t t_base, int n_chunk, const float* inv, int jb,
+                                               float& best, float& s_best, int& j_best) {
+    uint32_t va[16], vb[16];
+    ptx::tmem_ld_16cols(t_base, va);
+    for (int c0 = 0; c0 < n_chunk; c0 += 32) {
+        ptx::tmem_ld_wait(va);
+        const bool second = c0 + 16 < n_chunk;
+        if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
+        argmax16(va, inv + c0, jb + c0, best, s_best, j_best);
+        if (second) {
+            ptx::tmem_ld_wait(vb);
+            if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
+            argmax16(vb, inv + c0 + 16, jb + c0 + 16, best, s_best, j_best);
+        }
+    }
+}
+
+// What a score item leaves behind for one row: f, alpha and the row's count in the histograms of
+// the sort's row partition (a row block lies in block p0 of it and possibly p0 + 1).
+__device__ __forceinline__ void lf_finish_scores(const LinearForwardOut& out, int64_t b, int k, int64_t rb, int64_t row, int et,
+                                                 int j_best, float s_best, const float* s_inv2, int32_t* s_hist) {
+    const int64_t p0 = out.hist ? (rb * LF_TILE_M) / out.rows_per_block : 0;
+    if (row < b) {
+        store_index(out.f, out.f_type, row, j_best);
+        out.alpha[row] = s_best * s_inv2[j_best];
+        if (out.hist) atomicAdd(&s_hist[(int)(row / out.rows_per_block - p0) * k + j_best], 1);
+    }
+    ptx::named_barrier(1, 128);
+    if (out.hist) {
+        for (int j = et; j < 2 * k; j += 128) {
+            const int32_t c = s_hist[j];
+            if (c) atomicAdd(&out.hist[(p0 + j / k) * k + j % k], c);     // integers: exact in any order
+        }
+    }
+    ptx::named_barrier(1, 128);
+}
 
 __global__ void __launch_bounds__(LF_THREADS, 1)
 linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
@@ -243,40 +325,8 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t t_base = tmem_base + buf * (uint32_t)LF_TILE_N + lane_base;
-#pragma unroll 1
-                for (int sl = 0; sl < LF_TILE_N / 64; ++sl) {
-                    uint32_t v0[32], v1[32];
-                    ptx::tmem_ld_32x32(t_base + (uint32_t)(sl * 64), v0);
-                    ptx::tmem_ld_32x32(t_base + (uint32_t)(sl * 64 + 32), v1);
-                    ptx::tmem_ld_wait();
-                    if (sl == LF_TILE_N / 64 - 1) {          // the accumulator is in registers: hand it back
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
-                    }
-                    if (leader) ptx::bulk_wait_group_read<0>();     // the previous store has read the staging area
-                    ptx::named_barrier(1, 128);
-                    uint8_t* d0 = slab + row_in_tile * 128;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        *reinterpret_cast<uint4*>(d0 + ((c ^ (row_in_tile & 7)) << 4)) =
-                            make_uint4(pack_bf16(__uint_as_float(v0[8 * c]), __uint_as_float(v0[8 * c + 1])),
-                                       pack_bf16(__uint_as_float(v0[8 * c + 2]), __uint_as_float(v0[8 * c + 3])),
-                                       pack_bf16(__uint_as_float(v0[8 * c + 4]), __uint_as_float(v0[8 * c + 5])),
-                                       pack_bf16(__uint_as_float(v0[8 * c + 6]), __uint_as_float(v0[8 * c + 7])));
-                        *reinterpret_cast<uint4*>(d0 + (((c + 4) ^ (row_in_tile & 7)) << 4)) =
-                            make_uint4(pack_bf16(__uint_as_float(v1[8 * c]), __uint_as_float(v1[8 * c + 1])),
-                                       pack_bf16(__uint_as_float(v1[8 * c + 2]), __uint_as_float(v1[8 * c + 3])),
-                                       pack_bf16(__uint_as_float(v1[8 * c + 4]), __uint_as_float(v1[8 * c + 5])),
-                                       pack_bf16(__uint_as_float(v1[8 * c + 6]), __uint_as_float(v1[8 * c + 7])));
-                    }
-                    ptx::fence_proxy_async();
-                    ptx::named_barrier(1, 128);
-                    if (leader) {
-                        ptx::tma_store_2d(&tm_z, slab, (int32_t)(ct * LF_TILE_N + sl * 64), (int32_t)(rb * LF_TILE_M));
-                        ptx::bulk_commit_group();
-                    }
-                }
+                lf_store_z_tile(t_base, slab, row_in_tile, leader, &tm_z, (int32_t)(ct * LF_TILE_N), (int32_t)(rb * LF_TILE_M),
+                                [&] { if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]); });
             } else {
                 if (!norms_loaded) {      // C's norms come from the kernel in front
                     grid_dependency_wait();
@@ -294,40 +344,13 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
                     const uint32_t t_base = tmem_base + buf * (uint32_t)LF_TILE_N + lane_base;
-                    const int jb = ch * n_chunk;
-                    uint32_t va[16], vb[16];
-                    ptx::tmem_ld_16cols(t_base, va);
-                    for (int c0 = 0; c0 < n_chunk; c0 += 32) {
-                        ptx::tmem_ld_wait(va);
-                        const bool second = c0 + 16 < n_chunk;
-                        if (second) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 16), vb);
-                        argmax16(va, s_inv + jb + c0, jb + c0, best, s_best, j_best);
-                        if (second) {
-                            ptx::tmem_ld_wait(vb);
-                            if (c0 + 32 < n_chunk) ptx::tmem_ld_16cols(t_base + (uint32_t)(c0 + 32), va);
-                            argmax16(vb, s_inv + jb + c0 + 16, jb + c0 + 16, best, s_best, j_best);
-                        }
-                    }
+                    lf_score_chunk(t_base, n_chunk, s_inv + ch * n_chunk, ch * n_chunk, best, s_best, j_best);
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&s_tempty[buf]);
                 }
                 if (!ok) break;
-                // the sort's row partition: this row block lies in block p0 and possibly p0 + 1
-                const int64_t p0 = out.hist ? (rb * LF_TILE_M) / out.rows_per_block : 0;
-                if (row < b) {
-                    store_index(out.f, out.f_type, row, j_best);
-                    out.alpha[row] = s_best * s_inv2[j_best];
-                    if (out.hist) atomicAdd(&s_hist[(int)(row / out.rows_per_block - p0) * k + j_best], 1);
-                }
-                ptx::named_barrier(1, 128);
-                if (out.hist) {
-                    for (int j = et; j < 2 * k; j += 128) {
-                        const int32_t c = s_hist[j];
-                        if (c) atomicAdd(&out.hist[(p0 + j / k) * k + j % k], c);     // integers: exact in any order
-                    }
-                }
-                ptx::named_barrier(1, 128);
+                lf_finish_scores(out, b, k, rb, row, et, j_best, s_best, s_inv2, s_hist);
             }
         }
         if (leader) ptx::bulk_wait_group<0>();

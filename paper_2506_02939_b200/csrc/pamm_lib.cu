@@ -19,6 +19,7 @@
 #include "weight_grad_persist.cuh"
 #include "weight_grad_chunked.cuh"
 #include "linear_forward.cuh"
+#include "linear_forward_pair.cuh"
 #include "small_k.cuh"
 
 using namespace pamm;
@@ -649,8 +650,11 @@ pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n
         if (s != PAMM_OK) return s;
     }
     const LinearForwardOut out = {f, alpha, hist, (int)rpb, (int)f_type};
+    // pairs of CTAs on one 256-row tile wherever there are at least 256 rows; else one CTA per 128-row tile
+    const bool pairs = b >= LP_PAIR_M && sm_count() >= 2 && linear_forward_pair_plan_for(b, m, k, sm_count()).stages >= 2;
     prof_begin(PAMM_PROF_COMPRESS, st);
-    s = launch_linear_forward(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st);
+    s = pairs ? launch_linear_forward_pair(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st)
+              : launch_linear_forward(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st);
     prof_end(PAMM_PROF_COMPRESS, st);
     g_launches += 1;
     return s;
