@@ -590,7 +590,7 @@ def run_forward(args):
         "unit": "tokens/s", "n_gpus": 1, "steps": K, "warmup": 3, "ms_per_step": t_fused["median"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{w.name} forward: X bf16 b={b} n={n}, W n x m={m}, k={k}", "l2": "inputs exceed L2"},
-        "roofline": {"bound": "tensor", "kernel": "linear_forward_kernel (X [W | C^T], 128 x 256 tiles)", "achieved": tf,
+        "roofline": {"bound": "tensor", "kernel": "linear_forward_pair_kernel (X [W | C^T], 256 x 256 tiles on pairs of CTAs)", "achieved": tf,
                      "peak": peak_tf, "peak_source": f"of {peak_kind} (sustained bf16)", "unit": "TFLOP/s", "frac": tf / peak_tf,
                      "traffic": None, "algorithmic_flops": flops},
         "forward_ms": {"fused_product_and_compression": t_fused, "product_alone_same_kernel": t_prod,

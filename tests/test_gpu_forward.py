@@ -69,8 +69,12 @@ SMALL = [
     (1000, 136, 264, 17),
     (777, 520, 1032, 128),
     (2500, 200, 776, 300),
-    (129, 64, 8, 129),
+    (129, 64, 8, 129),          # fewer than 256 rows: one CTA per tile
+    (200, 200, 776, 48),        # the same, several column tiles
     (4133, 264, 520, 64),
+    (256, 64, 264, 129),        # exactly one pair of row blocks; generators padded to two halves of 80
+    (257, 136, 8, 33),          # the second pair holds one row
+    (640, 72, 520, 513),        # three chunks of generators on pairs of CTAs
 ]
 
 
