@@ -18,6 +18,7 @@
 #include "weight_grad_simt.cuh"
 #include "weight_grad_persist.cuh"
 #include "weight_grad_chunked.cuh"
+#include "compress_pair.cuh"
 #include "linear_forward.cuh"
 #include "linear_forward_pair.cuh"
 #include "small_k.cuh"
@@ -424,9 +425,13 @@ pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_d
                         const Neighbourhood& nb = NO_NEIGHBOURHOOD) {
     if (dt == PAMM_BF16 && compress_umma_usable(b, n, k, groups, sm_count(), nb.on)) {
         const CompressOut out = {f, alpha, out_stride, products, (int64_t)(sort_products_bytes(b, k) / 4), (int)f_type};
+        // many generators per chunk (tensor-bound): pairs of CTAs on one MMA tile; the same rows, results and counts
+        const bool pairs = !nb.on && compress_pair_usable(b, n, k, groups, sm_count());
         prof_begin(PAMM_PROF_COMPRESS, st);
-        const pamm_status s = launch_compress_umma(X, ldx, b, n, C, ldc, k, groups, c_invnorm, out, sm_count(), x_is_ready, st,
-                                                    nb.on, nb.eps, nb.dropped);
+        const pamm_status s = pairs
+            ? launch_compress_pair(X, ldx, b, n, C, ldc, k, groups, c_invnorm, out, sm_count(), x_is_ready, st)
+            : launch_compress_umma(X, ldx, b, n, C, ldc, k, groups, c_invnorm, out, sm_count(), x_is_ready, st, nb.on, nb.eps,
+                                   nb.dropped);
         prof_end(PAMM_PROF_COMPRESS, st);
         g_launches += 1;
         return s;
