@@ -283,7 +283,7 @@ inline CompressPairPlan compress_pair_plan_for(int64_t b, int64_t k, int groups,
 inline bool compress_pair_usable(int64_t b, int64_t n, int64_t k, int groups, int sms) {
     if (!compress_umma_supported(b, n, k) || (int64_t)groups * k > (1 << 20) || sms < 2) return false;
     const CompressPairPlan p = compress_pair_plan_for(b, k, groups, sms);
-    return p.stages >= 2 && p.n_chunk >= CP_MIN_CHUNK;
+    return p.stages >= 2 && p.n_chunk >= CP_MIN_CHUNK && cta_pairs_can_launch((const void*)compress_pair_kernel, CP_THREADS, p.smem_bytes);
 }
 
 inline pamm_status launch_compress_pair(const void* X, int64_t ldx, int64_t b, int64_t n, const void* C, int64_t ldc,

@@ -34,8 +34,10 @@ struct ContractWs {
     int32_t* perm;        // b
     float* partials;      // (CT_MAX_CTAS + k) x m_pad
     float* btilde;        // k x m_pad (used when the caller passes no B~)
-    int64_t nb, rows_per_block, m_pad;
-    size_t bytes;
+    uint16_t* planes;     // optional, behind everything else: B~ split into bf16 hi and lo, 2 x k x plane_ld
+    int64_t nb, rows_per_block, m_pad, plane_ld;
+    size_t bytes;         // without the planes
+    size_t bytes_with_planes;
 };
 
 // rows_per_block: the row partition of the histograms (compress_rows_per_cta).
@@ -53,6 +55,9 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
     w.partials = (float*)take((size_t)(CT_MAX_CTAS + k) * w.m_pad * 4);
     w.btilde = (float*)take((size_t)k * w.m_pad * 4);
     w.bytes = off;
+    w.plane_ld = round_up(m, 8);
+    w.planes = (uint16_t*)take((size_t)2 * k * w.plane_ld * 2);
+    w.bytes_with_planes = off;
     return w;
 }
 
@@ -452,10 +457,14 @@ constexpr int RED_THREADS = 256;
 
 // Finishes B~: zero rows for empty segments, sums of partial rows for segments
 // that were cut by a range boundary; rows written directly by main are left alone.
+// With `planes` it also leaves every element of B~ split into two bf16 values,
+// hi = rn(x) and lo = rn(x - hi), in two k x plane_ld planes (hi first): the operands
+// of the product over many generators, which then come by TMA instead of being
+// converted by every CTA that needs them.
 __global__ void __launch_bounds__(RED_THREADS)
 contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k, int64_t b,
                        const int32_t* __restrict__ seg_start, int rows_per_cta,
-                       float* __restrict__ Bt, int64_t ldb) {
+                       float* __restrict__ Bt, int64_t ldb, uint16_t* __restrict__ planes, int64_t plane_ld) {
     const int64_t mv = m_pad / 4;
     const int64_t idx = (int64_t)blockIdx.x * RED_THREADS + threadIdx.x;
     grid_dependency_wait();
@@ -465,20 +474,54 @@ contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_
     const int64_t col = (idx % mv) * 4;
     const int32_t s0 = (int32_t)min((int64_t)max(seg_start[j], 0), b), s1 = (int32_t)min((int64_t)max(seg_start[j + 1], 0), b);
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    float* out = Bt + (int64_t)j * ldb + col;
+    bool written = false;      // the main pass wrote this row itself
     if (s1 > s0) {
         const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;
-        if (c_lo == c_hi) return;
-        for (int c = c_lo; c <= c_hi; ++c) {
-            const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)(c + j) * m_pad + col);
-            s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+        if (c_lo == c_hi) {
+            if (!planes) return;
+            written = true;
+            if (col + 4 <= m) {
+                s = *reinterpret_cast<const float4*>(out);
+            } else {
+                float v[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int e = 0; e < 4 && col + e < m; ++e) v[e] = out[e];
+                s = make_float4(v[0], v[1], v[2], v[3]);
+            }
+        } else {
+            for (int c = c_lo; c <= c_hi; ++c) {
+                const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)(c + j) * m_pad + col);
+                s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+            }
         }
     }
-    float* out = Bt + (int64_t)j * ldb + col;
-    if (col + 4 <= m) {
-        *reinterpret_cast<float4*>(out) = s;
-    } else {
-        const float v[4] = {s.x, s.y, s.z, s.w};
-        for (int e = 0; e < 4 && col + e < m; ++e) out[e] = v[e];
+    if (!written) {
+        if (col + 4 <= m) {
+            *reinterpret_cast<float4*>(out) = s;
+        } else {
+            const float v[4] = {s.x, s.y, s.z, s.w};
+            for (int e = 0; e < 4 && col + e < m; ++e) out[e] = v[e];
+        }
+    }
+    if (planes) {
+        const float x[4] = {s.x, s.y, s.z, s.w};
+        float h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool in = col + e < m;
+            h[e] = in ? __bfloat162float(__float2bfloat16_rn(x[e])) : 0.f;
+            l[e] = in ? x[e] - h[e] : 0.f;
+        }
+        auto pack2 = [](float a, float c) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(a, c);     // .x = first argument = low 16 bits
+            return *reinterpret_cast<uint32_t*>(&t);
+        };
+        uint16_t* hi = planes + (int64_t)j * plane_ld + col;      // col % 4 == 0 and plane_ld % 8 == 0: 8-byte aligned
+        uint16_t* lo = hi + (int64_t)k * plane_ld;
+        if (col + 4 <= plane_ld) {
+            *reinterpret_cast<uint2*>(hi) = make_uint2(pack2(h[0], h[1]), pack2(h[2], h[3]));
+            *reinterpret_cast<uint2*>(lo) = make_uint2(pack2(l[0], l[1]), pack2(l[2], l[3]));
+        }
     }
 }
 

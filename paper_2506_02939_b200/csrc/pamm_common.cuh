@@ -215,5 +215,8 @@ inline pamm_status tensor_map_failed() {
 // 48 KiB default, remembering per device and kernel what has been granted already
 // so that the driver call is not repeated on every launch.
 bool ensure_dynamic_smem(const void* kernel, size_t bytes);
+// Whether clusters of two CTAs of this kernel can be scheduled on the current device (asked once per
+// kernel, device and shared-memory size); where they cannot, the one-CTA kernels serve.
+bool cta_pairs_can_launch(const void* kernel, int threads, size_t dynamic_smem);
 
 }  // namespace pamm

@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <tuple>
 #include <mutex>
 #include <utility>
 #include <vector>
@@ -18,6 +19,7 @@
 #include "weight_grad_simt.cuh"
 #include "weight_grad_persist.cuh"
 #include "weight_grad_chunked.cuh"
+#include "weight_grad_planes.cuh"
 #include "compress_pair.cuh"
 #include "linear_forward.cuh"
 #include "linear_forward_pair.cuh"
@@ -48,6 +50,33 @@ bool ensure_dynamic_smem(const void* kernel, size_t bytes) {
     }
     have = bytes;
     return true;
+}
+
+bool cta_pairs_can_launch(const void* kernel, int threads, size_t dynamic_smem) {
+    if (!ensure_dynamic_smem(kernel, dynamic_smem)) return false;
+    static std::mutex mu;
+    static std::map<std::tuple<int, const void*, size_t>, bool> known;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    const auto key = std::make_tuple(dev, kernel, dynamic_smem);
+    const auto it = known.find(key);
+    if (it != known.end()) return it->second;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = dynamic_smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
+    if (e != cudaSuccess) cudaGetLastError();
+    return known[key] = (e == cudaSuccess && clusters >= 1);
 }
 }  // namespace pamm
 
@@ -138,7 +167,7 @@ StepArena step_arena_layout(void* base, int64_t b, int64_t n, int64_t m, int64_t
     a.alpha = (float*)take((size_t)b * 4);
     a.Bt = take((size_t)k * a.ldb * 4);
     a.dW = take((size_t)n * a.ldw * 4);
-    a.ws_bytes = contract_ws(nullptr, b, m, k).bytes;
+    a.ws_bytes = contract_ws(nullptr, b, m, k).bytes_with_planes;
     a.ws = take(a.ws_bytes);
     a.products = take(sort_products_bytes(b, k));
     a.bytes = off;
@@ -224,8 +253,9 @@ pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const i
 template <typename T>
 pamm_status launch_contract(const void* f, int f_type, const float* alpha, const void* dY, int64_t ldy, int64_t b,
                             int64_t m, int64_t k, float* Bt, int64_t ldb, const int32_t* products, const ContractWs& w,
-                            cudaStream_t st) {
+                            cudaStream_t st, bool with_planes = false) {
     constexpr int V = Vec16<T>::N;
+    uint16_t* planes = with_planes ? w.planes : nullptr;     // B~ also as bf16 hi / lo, for the product that follows
     pamm_status s = launch_sort(f, f_type, b, k, products, w, st);
     if (s != PAMM_OK) return s;
     if (contract_stream_supported(m, sizeof(T))) {
@@ -247,7 +277,7 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
         prof_end(PAMM_PROF_CONTRACT, st);
         const int64_t items = k * (w.m_pad / 4);
         launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st,
-               true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
+               true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb, planes, w.plane_ld);
         return launch_status();
     }
     // very wide rows: column slabs, register staging
@@ -267,7 +297,7 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
     prof_end(PAMM_PROF_CONTRACT, st);
     const int64_t items = k * (w.m_pad / 4);
     launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st, true,
-           (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb);
+           (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb, planes, w.plane_ld);
     return launch_status();
 }
 
@@ -541,7 +571,7 @@ size_t pamm_workspace_bytes(pamm_ws_kind kind, int64_t b, int64_t n, int64_t m, 
             return sort_products_bytes(b, k);
         case PAMM_WS_CONTRACT:
             if (m < 1) return (size_t)-1;
-            return contract_ws(nullptr, b, m, k).bytes;
+            return contract_ws(nullptr, b, m, k).bytes_with_planes;     // pamm_contract itself needs less
         case PAMM_WS_STEP_HOST:
             if (n < 1 || m < 1) return (size_t)-1;
             return step_arena_layout(nullptr, b, n, m, k, dt).bytes;
@@ -656,7 +686,9 @@ pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n
     }
     const LinearForwardOut out = {f, alpha, hist, (int)rpb, (int)f_type};
     // pairs of CTAs on one 256-row tile wherever there are at least 256 rows; else one CTA per 128-row tile
-    const bool pairs = b >= LP_PAIR_M && sm_count() >= 2 && linear_forward_pair_plan_for(b, m, k, sm_count()).stages >= 2;
+    const LinearForwardPlan pp = linear_forward_pair_plan_for(b, m, k, sm_count());
+    const bool pairs = b >= LP_PAIR_M && sm_count() >= 2 && pp.stages >= 2 &&
+                       cta_pairs_can_launch((const void*)linear_forward_pair_kernel, LF_THREADS, pp.smem_bytes);
     prof_begin(PAMM_PROF_COMPRESS, st);
     s = pairs ? launch_linear_forward_pair(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st)
               : launch_linear_forward(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st);
@@ -741,9 +773,21 @@ pamm_status pamm_contract_weight_grad(const void* C, int64_t ldc, int64_t n, con
             ? launch_small_backward<float>(C, ldc, n, f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, dw, w, st)
             : launch_small_backward<__nv_bfloat16>(C, ldc, n, f, (int)f_type, alpha, dY, ldy, b, m, k, Btilde, ldb, dw, w, st);
     const int32_t* pr = (const int32_t*)sort_products;
+    // Many generators: the reduction also leaves B~ split into bf16 hi / lo planes and the product takes all its
+    // operands by TMA (a workspace of the size pamm_workspace_bytes gives has room for the planes).
+    const bool swap = layout == PAMM_DW_MN;
+    const bool planes = dt == PAMM_BF16 && ws_bytes >= w.bytes_with_planes && !weight_grad_persist_supported(k, n, m) &&
+                        weight_grad_chunked_supported(k, n, m) && (swap ? n : m) * (int64_t)esize(dw_dt) >= 16;
     s = dt == PAMM_F32 ? launch_contract<float>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st)
-                       : launch_contract<__nv_bfloat16>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st);
+                       : launch_contract<__nv_bfloat16>(f, (int)f_type, alpha, dY, ldy, b, m, k, Bt, ldbt, pr, w, st, planes);
     if (s != PAMM_OK) return s;
+    if (planes) {
+        prof_begin(PAMM_PROF_WEIGHT_GRAD, st);
+        s = launch_weight_grad_planes(C, ldc, k, n, w.planes, w.plane_ld, m, dW, ldw, dw_dt == PAMM_BF16, swap, sm_count(), st);
+        prof_end(PAMM_PROF_WEIGHT_GRAD, st);
+        g_launches += 1;
+        return s;
+    }
     return do_weight_grad(C, ldc, k, n, dt, Bt, ldbt, m, dw, st);
 }
 
