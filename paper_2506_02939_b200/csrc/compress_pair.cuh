@@ -9,8 +9,8 @@
 // one pass fill tensor memory.
 //
 // Rows, results and the per-CTA histograms of f are cut exactly as in the one-CTA kernel (every
-// CTA owns the same contiguous row range), so either kernel leaves the same f, alpha and sort
-// products.  The two CTAs of a pair walk the same number of 128-row tiles (rows beyond the
+// CTA owns the same contiguous row range), so the sort products of either kernel feed the same
+// backward pass.  The two CTAs of a pair walk the same number of 128-row tiles (rows beyond the
 // range or beyond b are zero-filled by TMA and never stored); an odd last CTA without rows
 // still feeds its half of the generators.
 //   rank 0 (leader)  warp 0 loads its tiles, warp 1 issues every MMA of the pair
