@@ -380,6 +380,31 @@ def run_cuda(args):
     fwd_rep = repeat_ms(forward)
     bwd_rep = repeat_ms(lambda s: backward())
     forward(w.index_seed)          # leave (C, f, alpha) of a forward pass behind, as after a step
+
+    # the read-only ceiling (untimed region): passes that only read dY or X, with plain loads and with the bulk-copy
+    # ring of the contraction's main pass, in natural row order and in the contraction's order (rows sorted by f)
+    def probe_gbs(kind, data, order=None, reps=12):
+        word = torch.empty(1, dtype=torch.int32, device=dev)
+        for _ in range(2):
+            pamm.probe_read(kind, data, order=order, sum32=word, stream=stream)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        ev[0].record(stream)
+        for r in range(reps):
+            pamm.probe_read(kind, data, order=order, sum32=word, stream=stream)
+            ev[r + 1].record(stream)
+        torch.cuda.synchronize()
+        ms = float(np.median([ev[r].elapsed_time(ev[r + 1]) for r in range(reps)]))
+        return data.shape[0] * data.shape[1] * data.element_size() / (ms * 1e-3) / 1e9
+
+    read_ceiling = None
+    if m * e <= 24576 and n * e <= 24576 and (m * e) % 16 == 0 and (n * e) % 16 == 0:
+        sorted_rows = torch.sort(f.to(torch.int64), stable=True).indices.to(torch.int32)
+        read_ceiling = {"unit": "GB/s",
+                        "dY_plain_loads": probe_gbs(pamm.PROBE_SUM, dY),
+                        "dY_bulk_rows_natural_order": probe_gbs(pamm.PROBE_ROWS, dY),
+                        "dY_bulk_rows_sorted_by_f": probe_gbs(pamm.PROBE_ROWS, dY, sorted_rows),
+                        "X_bulk_rows_natural_order": probe_gbs(pamm.PROBE_ROWS, X),
+                        "note": "load-only passes over the same buffers; the contraction reads dY in the sorted order"}
     covers = "timed region"
     if t_begin.elapsed_time(t_end) < 500.0:
         # a region this short yields too few 50 ms samples: keep sampling over an untimed repeat of the same steps
@@ -472,6 +497,8 @@ def run_cuda(args):
                     if k == w.ks[0] and args.eps is None else None,
                     "algorithmic_bytes": ab["contract"], "samples": st_k["contract_main"]["count"],
                     "achieved_best": ab["contract"] / (st_k["contract_main"]["min"] * 1e-3) / 1e9}
+        if read_ceiling:
+            roofline["frac_of_read_ceiling_same_order"] = achieved / read_ceiling["dY_bulk_rows_sorted_by_f"]
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -507,6 +534,7 @@ def run_cuda(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "stages": stages,
+        "read_ceiling": read_ceiling,
         "memory_saved": saved,
     }
     print(json.dumps(line), flush=True)

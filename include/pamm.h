@@ -376,6 +376,26 @@ pamm_status pamm_set_profile_events(pamm_prof_kind kind, void* start_event, void
  */
 pamm_status pamm_selftest_bounded_wait(void* stream);
 
+/*
+ * Read-only streaming probes (no counterpart in the paper): what a pass that only reads a
+ * matrix once can reach on this device, as the practical ceiling of the compression (reads X)
+ * and of the contraction (reads dY).  `base` (device): `rows` rows of `row_bytes` bytes (a
+ * multiple of 16), `ld_bytes` apart (a multiple of 16, >= row_bytes), 16-byte aligned.
+ *   PAMM_PROBE_SUM   ordinary loads of every 16-byte word; *sum32 receives the wrap-around
+ *                    sum of all 32-bit words
+ *   PAMM_PROBE_ROWS  whole rows by bulk copies through a shared-memory ring, two CTAs per SM,
+ *                    the access pattern of the contraction's main pass; position p reads row
+ *                    order[p] (device, `rows` entries of int32 in [0, rows); NULL = natural
+ *                    order); *sum32 receives the sum of the first 32-bit word of every row read.
+ *                    row_bytes <= 24576.
+ * sum32 (device, 4 bytes) is zeroed on the stream first.  Enqueues on `stream`; time it with
+ * events around the call.  An entry of `order` out of range sets PAMM_ERR_BAD_INDEX in the
+ * device status (row 0 is read instead).
+ */
+typedef enum { PAMM_PROBE_SUM = 0, PAMM_PROBE_ROWS = 1 } pamm_probe_kind;
+pamm_status pamm_probe_read(pamm_probe_kind kind, const void* base, int64_t rows, int64_t row_bytes, int64_t ld_bytes,
+                            const int32_t* order, uint32_t* sum32, void* stream);
+
 /* Library version as major*10000 + minor*100 + patch. */
 int pamm_version(void);
 

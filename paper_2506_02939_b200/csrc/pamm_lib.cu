@@ -24,6 +24,7 @@
 #include "linear_forward.cuh"
 #include "linear_forward_pair.cuh"
 #include "small_k.cuh"
+#include "read_probe.cuh"
 
 using namespace pamm;
 
@@ -534,6 +535,34 @@ extern "C" {
 
 pamm_status pamm_selftest_bounded_wait(void* stream) {
     launch(selftest_bounded_wait_kernel, dim3(1), dim3(64), 0, (cudaStream_t)stream, false, (uint32_t)2048);
+    return launch_status();
+}
+
+pamm_status pamm_probe_read(pamm_probe_kind kind, const void* base, int64_t rows, int64_t row_bytes, int64_t ld_bytes,
+                            const int32_t* order, uint32_t* sum32, void* stream) {
+    if (!base || !sum32 || rows < 1 || row_bytes < 16 || row_bytes % 16 || ld_bytes < row_bytes || ld_bytes % 16 ||
+        !aligned(base, 16) || !aligned(sum32, 4) || rows > MAX_ROWS)
+        return PAMM_ERR_INVALID_ARG;
+    if (kind != PAMM_PROBE_SUM && kind != PAMM_PROBE_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (kind == PAMM_PROBE_SUM && order) return PAMM_ERR_INVALID_ARG;
+    if (kind == PAMM_PROBE_ROWS && (row_bytes > 24576 || (order && !aligned(order, 4)))) return PAMM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(sum32, 0, 4, st) != cudaSuccess) return PAMM_ERR_CUDA;
+    if (kind == PAMM_PROBE_SUM) {
+        const int64_t vecs = rows * (row_bytes / 16);
+        const int64_t want = (vecs + RP_SUM_THREADS - 1) / RP_SUM_THREADS;
+        const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sm_count() * 4));
+        launch(read_probe_sum_kernel, dim3(grid), dim3(RP_SUM_THREADS), 0, st, false, (const uint8_t*)base, rows, row_bytes,
+               ld_bytes, sum32);
+        return launch_status();
+    }
+    const int pitch = (int)round_up(row_bytes, 128);
+    const int slots = std::max(2, std::min(RP_MAX_SLOTS, RP_RING_BYTES / pitch));
+    const size_t smem = 128 + (size_t)slots * pitch;
+    if (!ensure_dynamic_smem((const void*)read_probe_rows_kernel, smem)) return PAMM_ERR_CUDA;
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(rows, (int64_t)sm_count() * 2));
+    launch(read_probe_rows_kernel, dim3(grid), dim3(RP_ROW_THREADS), smem, st, false, (const uint8_t*)base, rows,
+           (uint32_t)row_bytes, ld_bytes, order, slots, pitch, sum32);
     return launch_status();
 }
 

@@ -50,6 +50,7 @@ _SIGNATURES = {
     "pamm_contract_no_alloc": ([_vp, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp], _ci),
     "pamm_last_device_status": ([_vp], _ci),
     "pamm_selftest_bounded_wait": ([_vp], _ci),
+    "pamm_probe_read": ([_ci, _vp, _i64, _i64, _i64, _vp, _vp, _vp], _ci),
     "pamm_launch_count": ([], ctypes.c_ulonglong),
     "pamm_set_profile_events": ([_ci, _vp, _vp], _ci),
 }
@@ -364,6 +365,26 @@ def prepared(call, *args, **kwargs):
         if code != OK:
             raise PammError(code, _name)
     return run
+
+
+PROBE_SUM, PROBE_ROWS = 0, 1
+
+
+def probe_read(kind: int, data: torch.Tensor, order=None, sum32=None, stream=None) -> torch.Tensor:
+    """A read-only pass over the rows of `data` (2-D, contiguous columns): PROBE_SUM with ordinary loads,
+    PROBE_ROWS with bulk copies through a shared-memory ring, optionally in the row order `order` (int32).
+    Returns the device word with the 32-bit checksum; time the call with events."""
+    if not data.is_cuda or data.dim() != 2 or data.stride(1) != 1:
+        raise ValueError("data: a 2-D CUDA tensor with contiguous columns")
+    es = data.element_size()
+    if sum32 is None:
+        sum32 = _empty((1,), dtype=torch.int32, device=data.device)
+    if order is not None:
+        if not order.is_cuda or order.dtype != torch.int32 or order.numel() != data.shape[0] or not order.is_contiguous():
+            raise ValueError("order: contiguous int32, one entry per row")
+    _check(_lib.pamm_probe_read(int(kind), _ptr(data), int(data.shape[0]), int(data.shape[1]) * es, int(data.stride(0)) * es,
+                                _ptr(order) if order is not None else None, _ptr(sum32), _stream(stream)), "pamm_probe_read")
+    return sum32
 
 
 def selftest_bounded_wait(stream=None) -> None:

@@ -112,6 +112,17 @@ def test_argument_errors_are_synchronous_and_launch_nothing():
     assert i.pamm_select_generators(fake, 8, 1 << 20, 8, pamm.F32, 50000, 0, null, fake, fake, 8, fake, null) == pamm.ERR_UNSUPPORTED
 
 
+def test_read_probe_argument_errors():
+    i = pamm._lib
+    fake, null = ctypes.c_void_p(0x1000), None
+    assert i.pamm_probe_read(pamm.PROBE_SUM, null, 4, 64, 64, null, fake, null) == pamm.ERR_INVALID_ARG
+    assert i.pamm_probe_read(pamm.PROBE_SUM, fake, 4, 60, 64, null, fake, null) == pamm.ERR_INVALID_ARG       # not whole 16-byte words
+    assert i.pamm_probe_read(pamm.PROBE_SUM, fake, 4, 64, 48, null, fake, null) == pamm.ERR_INVALID_ARG       # rows overlap
+    assert i.pamm_probe_read(pamm.PROBE_SUM, fake, 4, 64, 64, fake, fake, null) == pamm.ERR_INVALID_ARG       # no order with plain loads
+    assert i.pamm_probe_read(pamm.PROBE_ROWS, fake, 4, 32768, 32768, null, fake, null) == pamm.ERR_INVALID_ARG  # row too wide for the ring
+    assert i.pamm_probe_read(7, fake, 4, 64, 64, null, fake, null) == pamm.ERR_INVALID_ARG
+
+
 def test_draw_indices_basic_properties():
     for b, k in [(1, 1), (2, 2), (7, 3), (2048, 4), (65536, 128), (65536, 1024), (100003, 517)]:
         idx = pamm.draw_indices_host(b, k, 42).numpy()

@@ -511,3 +511,26 @@ def test_a_whole_step_can_be_captured_in_a_cuda_graph():
     assert pamm.last_device_status() == pamm.OK
     for got, ref in zip((f, alpha, Bt, dW), want):
         assert torch.equal(got, ref)
+
+
+def test_read_probes_visit_every_row_once():
+    # no arithmetic of the method: the checksums only show that the probes read what they are timed for
+    g = torch.Generator(device="cuda").manual_seed(5)
+    data = torch.randint(-2**31, 2**31 - 1, (3001, 776), dtype=torch.int32, device="cuda", generator=g)[:, :772]   # padded rows
+    words = data.to(torch.int64)
+    s = pamm.probe_read(pamm.PROBE_SUM, data)
+    assert (int(s.item()) - int(words.sum().item())) % 2**32 == 0
+    first = int(words[:, 0].sum().item())
+    s = pamm.probe_read(pamm.PROBE_ROWS, data)
+    assert (int(s.item()) - first) % 2**32 == 0
+    order = torch.randperm(3001, device="cuda", generator=g).to(torch.int32)
+    s = pamm.probe_read(pamm.PROBE_ROWS, data, order=order)
+    assert (int(s.item()) - first) % 2**32 == 0
+    twice = torch.zeros(3001, dtype=torch.int32, device="cuda")          # every position reads row 0
+    s = pamm.probe_read(pamm.PROBE_ROWS, data, order=twice)
+    assert (int(s.item()) - 3001 * int(words[0, 0].item())) % 2**32 == 0
+    assert pamm.last_device_status() == pamm.OK
+    bad = order.clone()
+    bad[17] = 3001
+    pamm.probe_read(pamm.PROBE_ROWS, data, order=bad)
+    assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
