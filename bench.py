@@ -606,6 +606,9 @@ def run_forward(args):
     t_prod = timed(product_alone, K)
     t_comp = timed(compress_alone, K)
     t_torch = timed(torch_gemm, K)
+    dX = torch.empty((b, n), dtype=torch.bfloat16, device=dev)
+    t_dx = timed(lambda s: pamm.linear_backward_input(Z, W, dX=dX, stream=stream), K)     # Algorithm 3's dX = dZ W^T, dZ := Z
+    t_dx_torch = timed(lambda s: torch.matmul(Z, W.t(), out=dX), K)
     clocks = sampler.stop()
     status = pamm.last_device_status()
     if status != pamm.OK:
@@ -624,7 +627,8 @@ def run_forward(args):
         "forward_ms": {"fused_product_and_compression": t_fused, "product_alone_same_kernel": t_prod,
                        "compression_alone": t_comp,
                        "cost_of_compression_inside_the_product_ms": t_fused["median"] - t_prod["median"],
-                       "torch_matmul_context_only": t_torch},
+                       "torch_matmul_context_only": t_torch,
+                       "input_gradient_product_dZ_Wt": t_dx, "torch_matmul_dZ_Wt_context_only": t_dx_torch},
         "gpu_launches": int(launches), "clocks": clocks,
     }
     print(json.dumps(line), flush=True)

@@ -174,6 +174,17 @@ pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n
                                 void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * The other product of the layer's backward pass (Algorithm 3: "grad X = grad Z W^T"), through the
+ * same tensor-core kernel as pamm_linear_forward: dX (b x n) = dZ (b x m) W^T with W (n x m) the
+ * layer's weight exactly as the forward pass takes it (here it is the operand whose contraction
+ * index, m, is contiguous).  bf16 only (PAMM_ERR_UNSUPPORTED otherwise); pointers are device
+ * pointers, 16-byte aligned, leading dimensions in elements (multiples of 8).  It does not share
+ * the read of dZ with the contraction: pamm_contract_weight_grad reads dZ once more.
+ */
+pamm_status pamm_linear_backward_input(const void* dZ, int64_t lddz, int64_t b, int64_t m, const void* W, int64_t ldw,
+                                       int64_t n, pamm_dtype dt, void* dX, int64_t lddx, void* stream);
+
+/*
  * Step 2 for several generator sets at once -- one compression per projection
  * (Section 4: the method "is applied to the Q, K and V projections"; the worked
  * example of the appendix "Complexity Analysis" has m = n per projection) -- in ONE

@@ -5,7 +5,8 @@ of the CUDA library (``pamm_linear_forward``: the scores are extra output column
 product, so X is not read a second time); other dtypes take torch's GEMM for Z and the
 library's stand-alone compression.  The layer saves (C, f, alpha, W) and lets go of X.
 Backward: the weight gradient is ``ApproxMM(C, alpha, f, dZ) = C^T B~`` through the library,
-the input gradient ``dX = dZ W^T`` is exact (torch).  Meant for the fused Q|K|V projection: ``W`` is n x m
+the input gradient ``dX = dZ W^T`` is exact (for bf16 layers the library's tensor-core product
+``pamm_linear_backward_input``, else torch).  Meant for the fused Q|K|V projection: ``W`` is n x m
 with m = |Q| + |K| + |V|, as in the paper's notation.
 """
 from __future__ import annotations
@@ -53,7 +54,17 @@ class PammLinearFunction(torch.autograd.Function):
     def backward(ctx, dZ):
         C, f, alpha, sp, W = ctx.saved_tensors
         n, m = W.shape
-        dX = dZ @ W.t() if ctx.needs_input_grad[0] else None
+        dX = None
+        if ctx.needs_input_grad[0]:
+            Wd = W.detach()
+            dZr = _rows(dZ, m)
+            own = (dZr.dtype == torch.bfloat16 and Wd.dtype == torch.bfloat16 and n >= 8 and m >= 8 and Wd.is_contiguous()
+                   and dZr.stride(1) == 1 and (m * 2) % 16 == 0 and (dZr.stride(0) * 2) % 16 == 0
+                   and Wd.data_ptr() % 16 == 0 and dZr.data_ptr() % 16 == 0)
+            if own:      # Algorithm 3's other product, through the library's tensor-core kernel
+                dX = pamm.linear_backward_input(dZr, Wd).reshape(*dZ.shape[:-1], n)
+            else:
+                dX = dZ @ W.t()
         dW = None
         if ctx.needs_input_grad[1]:
             dZ2 = _rows(dZ.to(C.dtype), m)

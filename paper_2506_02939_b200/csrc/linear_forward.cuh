@@ -176,7 +176,7 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                       const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_z,
                       int64_t b, int n, int m, int k, int n_chunk, int num_chunks, int stages,
                       int64_t row_blocks, int64_t col_tiles, int64_t items,
-                      const float* __restrict__ c_invnorm, LinearForwardOut out) {
+                      const float* __restrict__ c_invnorm, LinearForwardOut out, int w_kmajor) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t s_full[8], s_empty[8], s_tfull[2], s_tempty[2];
     __shared__ uint32_t s_tmem_base;
@@ -239,6 +239,8 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                         ptx::tma_load_2d(stage, &tm_x, ks * LF_BLOCK_K, (int32_t)(rb * LF_TILE_M), &s_full[s]);
                         if (score) {
                             ptx::tma_load_2d(stage + LF_A_BYTES, &tm_c, ks * LF_BLOCK_K, u * n_chunk, &s_full[s]);
+                        } else if (w_kmajor) {      // W given as columns x hidden: the tile's 256 columns are 256 rows of it
+                            ptx::tma_load_2d(stage + LF_A_BYTES, &tm_w, ks * LF_BLOCK_K, (int32_t)(ct * LF_TILE_N), &s_full[s]);
                         } else {
 #pragma unroll
                             for (int q = 0; q < 4; ++q)
@@ -263,7 +265,7 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (ptx::elect_one()) {
-            const uint32_t idesc_z = ptx::umma_idesc_bf16(LF_TILE_M, LF_TILE_N) | (1u << 16);     // B (W) is MN-major
+            const uint32_t idesc_z = ptx::umma_idesc_bf16(LF_TILE_M, LF_TILE_N) | (w_kmajor ? 0u : 1u << 16);   // bit 16: B (W) MN-major
             const uint32_t idesc_s = ptx::umma_idesc_bf16(LF_TILE_M, (uint32_t)n_chunk);          // B (C) is K-major
             uint32_t unit = 0, sph = 0;
             int s = 0;               // ring stage and the parity of its use
@@ -284,11 +286,12 @@ linear_forward_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_con
                         const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)s * LF_STAGE_BYTES);
                         const uint32_t b_addr = a_addr + LF_A_BYTES;
                         const uint64_t desc_a = ptx::umma_desc_k_sw128(a_addr);
-                        if (score) {
+                        if (score || w_kmajor) {
                             const uint64_t desc_b = ptx::umma_desc_k_sw128(b_addr);
+                            const uint32_t idesc = score ? idesc_s : idesc_z;
 #pragma unroll
                             for (int kk = 0; kk < LF_BLOCK_K / 16; ++kk)
-                                ptx::umma_bf16(d_addr, desc_a + 2 * kk, desc_b + 2 * kk, idesc_s, (ks | kk) != 0);
+                                ptx::umma_bf16(d_addr, desc_a + 2 * kk, desc_b + 2 * kk, idesc, (ks | kk) != 0);
                         } else {
 #pragma unroll
                             for (int kk = 0; kk < LF_BLOCK_K / 16; ++kk)   // 16 hidden indices = two 8-deep groups = 2048 bytes
@@ -380,12 +383,14 @@ inline LinearForwardPlan linear_forward_plan_for(int64_t b, int64_t m, int64_t k
 
 inline pamm_status launch_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n, const void* W, int64_t ldw,
                                          int64_t m, const void* C, int64_t ldc, int64_t k, const float* c_invnorm,
-                                         void* Z, int64_t ldz, const LinearForwardOut& out, int sms, cudaStream_t st) {
+                                         void* Z, int64_t ldz, const LinearForwardOut& out, int sms, cudaStream_t st,
+                                         bool w_kmajor = false) {
     const LinearForwardPlan p = linear_forward_plan_for(b, m, k, sms);
     if (p.stages < 2) return PAMM_ERR_UNSUPPORTED;
     CUtensorMap tm_x, tm_w, tm_c, tm_z;
     if (!make_tmap_bf16_sw128(&tm_x, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, LF_TILE_M) ||
-        !make_tmap_bf16_sw128(&tm_w, W, (uint64_t)n, (uint64_t)m, (uint64_t)ldw, LF_BLOCK_K) ||
+        !(w_kmajor ? make_tmap_bf16_sw128(&tm_w, W, (uint64_t)m, (uint64_t)n, (uint64_t)ldw, LF_TILE_N)      // m x n: columns x hidden
+                   : make_tmap_bf16_sw128(&tm_w, W, (uint64_t)n, (uint64_t)m, (uint64_t)ldw, LF_BLOCK_K)) ||
         !(k > 0 ? make_tmap_bf16_sw128(&tm_c, C, (uint64_t)k, (uint64_t)n, (uint64_t)ldc, (uint32_t)p.n_chunk)
                 : make_tmap_bf16_sw128(&tm_c, X, (uint64_t)b, (uint64_t)n, (uint64_t)ldx, LF_TILE_M)) ||     // unused without generators
         !make_tmap_bf16_sw128(&tm_z, Z, (uint64_t)b, (uint64_t)m, (uint64_t)ldz, LF_TILE_M))
@@ -402,7 +407,7 @@ inline pamm_status launch_linear_forward(const void* X, int64_t ldx, int64_t b, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, linear_forward_kernel, tm_x, tm_w, tm_c, tm_z, b, (int)n, (int)m, (int)k, p.n_chunk, p.num_chunks,
-                       p.stages, p.row_blocks, p.col_tiles, p.items, c_invnorm, out);
+                       p.stages, p.row_blocks, p.col_tiles, p.items, c_invnorm, out, w_kmajor ? 1 : 0);
     return launch_result("linear_forward_kernel launch");
 }
 

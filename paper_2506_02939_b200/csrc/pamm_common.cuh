@@ -206,10 +206,7 @@ inline pamm_status launch_result(const char* what) {
     return PAMM_ERR_CUDA;
 }
 
-inline pamm_status tensor_map_failed() {
-    note_cuda_failure("cuTensorMapEncodeTiled (tensor map of an operand)", cudaErrorInvalidValue);
-    return PAMM_ERR_CUDA;
-}
+pamm_status tensor_map_failed();     // notes what the failed encoding was asked for
 
 // Raises a kernel's dynamic shared-memory limit when a launch needs more than the
 // 48 KiB default, remembering per device and kernel what has been granted already

@@ -34,6 +34,16 @@ void note_cuda_failure(const char* what, cudaError_t err) {
     snprintf(g_cuda_detail, sizeof g_cuda_detail, "%s: %s (%s)", what, cudaGetErrorName(err), cudaGetErrorString(err));
 }
 
+pamm_status tensor_map_failed() {
+    const TmapFailure& f = last_tmap_failure();
+    snprintf(g_cuda_detail, sizeof g_cuda_detail,
+             "cuTensorMapEncodeTiled failed (CUresult %d; no driver entry point if 0) for a %llu x %llu matrix of %u-byte elements "
+             "at %p, leading dimension %llu, boxes of %u rows",
+             f.result, (unsigned long long)f.rows, (unsigned long long)f.cols, f.elem_bytes, f.base, (unsigned long long)f.ld,
+             f.box_rows);
+    return PAMM_ERR_CUDA;
+}
+
 bool ensure_dynamic_smem(const void* kernel, size_t bytes) {
     if (bytes <= 48 * 1024) return true;
     static std::mutex mu;
@@ -722,6 +732,27 @@ pamm_status pamm_linear_forward(const void* X, int64_t ldx, int64_t b, int64_t n
     s = pairs ? launch_linear_forward_pair(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st)
               : launch_linear_forward(X, ldx, b, n, W, ldw, m, C, ldc, k, c_invnorm, Z, ldz, out, sm_count(), st);
     prof_end(PAMM_PROF_COMPRESS, st);
+    g_launches += 1;
+    return s;
+}
+
+pamm_status pamm_linear_backward_input(const void* dZ, int64_t lddz, int64_t b, int64_t m, const void* W, int64_t ldw,
+                                       int64_t n, pamm_dtype dt, void* dX, int64_t lddx, void* stream) {
+    if (!dtype_ok(dt)) return PAMM_ERR_UNSUPPORTED;
+    if (!dZ || !W || !dX || b < 1 || n < 1 || m < 1 || b > MAX_ROWS) return PAMM_ERR_INVALID_ARG;
+    if (!ld_ok(lddz, m, esize(dt)) || !ld_ok(ldw, m, esize(dt)) || !ld_ok(lddx, n, esize(dt))) return PAMM_ERR_INVALID_ARG;
+    if (!aligned(dZ, 16) || !aligned(W, 16) || !aligned(dX, 16)) return PAMM_ERR_INVALID_ARG;
+    // the forward kernel with the roles renamed: rows of dZ, contraction over m, n output columns, W as columns x hidden
+    if (dt != PAMM_BF16 || !linear_forward_supported(b, m, n, 0) || linear_forward_plan_for(b, n, 0, sm_count()).stages < 2)
+        return PAMM_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const LinearForwardOut out = {nullptr, nullptr, nullptr, 1, (int)PAMM_IDX_I32};
+    const LinearForwardPlan pp = linear_forward_pair_plan_for(b, n, 0, sm_count());
+    const bool pairs = b >= LP_PAIR_M && sm_count() >= 2 && pp.stages >= 2 &&
+                       cta_pairs_can_launch((const void*)linear_forward_pair_kernel, LF_THREADS, pp.smem_bytes);
+    const pamm_status s = pairs
+        ? launch_linear_forward_pair(dZ, lddz, b, m, W, ldw, n, nullptr, 0, 0, nullptr, dX, lddx, out, sm_count(), st, true)
+        : launch_linear_forward(dZ, lddz, b, m, W, ldw, n, nullptr, 0, 0, nullptr, dX, lddx, out, sm_count(), st, true);
     g_launches += 1;
     return s;
 }

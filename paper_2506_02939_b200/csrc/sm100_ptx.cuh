@@ -287,6 +287,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 inline EncodeTiledFn encode_tiled_fn() {
+    // The driver call needs a current context.  A thread that has made no context-binding runtime call yet
+    // (a framework's worker thread whose first library call goes straight to an encoding) has none:
+    // cudaFree(0) binds the device's primary context to the thread, once.
+    static thread_local bool context_bound = false;
+    if (!context_bound) {
+        cudaFree(0);
+        context_bound = true;
+    }
     static EncodeTiledFn fn = nullptr;
     static bool tried = false;
     if (!tried) {
@@ -300,6 +308,18 @@ inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// What the last failed encoding on this thread was asked for (for the error detail).
+struct TmapFailure {
+    const void* base;
+    uint64_t rows, cols, ld;
+    uint32_t box_rows, elem_bytes;
+    int result;
+};
+inline TmapFailure& last_tmap_failure() {
+    static thread_local TmapFailure f = {nullptr, 0, 0, 0, 0, 0, 0};
+    return f;
+}
+
 // Row-major bf16 matrix (rows x cols, leading dimension ld elements) tiled in
 // boxes of box_rows x 64 columns with the 128-byte swizzle; out-of-range
 // elements read as zero.
@@ -311,9 +331,11 @@ inline bool make_tmap_bf16_sw128(CUtensorMap* tm, const void* base, uint64_t row
     cuuint64_t strides[1] = {ld * 2};
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) last_tmap_failure() = {base, rows, cols, ld, box_rows, 2u, (int)r};
+    return r == CUDA_SUCCESS;
 }
 
 // Row-major fp32 matrix tiled in boxes of box_rows x 32 columns (128 bytes), 128-byte swizzle.
@@ -325,9 +347,11 @@ inline bool make_tmap_f32_sw128(CUtensorMap* tm, const void* base, uint64_t rows
     cuuint64_t strides[1] = {ld * 4};
     cuuint32_t box[2] = {32, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) last_tmap_failure() = {base, rows, cols, ld, box_rows, 4u, (int)r};
+    return r == CUDA_SUCCESS;
 }
 
 }  // namespace pamm

@@ -39,6 +39,7 @@ _SIGNATURES = {
     "pamm_compress_projections": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _i64, _vp, _vp, _ci, _vp, _i64, _vp, _sz, _vp], _ci),
     "pamm_linear_forward": ([_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _i64, _u64, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _vp, _ci,
                              _vp, _vp, _sz, _vp], _ci),
+    "pamm_linear_backward_input": ([_vp, _i64, _i64, _i64, _vp, _i64, _i64, _ci, _vp, _i64, _vp], _ci),
     "pamm_contract": ([_vp, _ci, _vp, _vp, _i64, _i64, _i64, _ci, _i64, _vp, _i64, _vp, _vp, _sz, _vp], _ci),
     "pamm_weight_grad": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, _i64, _ci, _ci, _vp], _ci),
     "pamm_compress_eps": ([_vp, _i64, _i64, _i64, _ci, _vp, _i64, _i64, _vp, ctypes.c_float, _vp, _ci, _vp, _vp, _vp, _sz, _vp], _ci),
@@ -274,6 +275,16 @@ def linear_forward(X, W, k: int, seed: int = 0, idx_in=None, Z=None, idx_out=Non
                                     _ptr(C), _ld(C), _ptr(c_invnorm), _ptr(Z), _ld(Z), _ptr(f), _ft(f), _ptr(alpha),
                                     _ptr(sort_products), _bytes(sort_products), _stream(stream)), "pamm_linear_forward")
     return Z, idx_out, C, c_invnorm, f, alpha
+
+
+def linear_backward_input(dZ, W, dX=None, stream=None):
+    """Algorithm 3's other product through the same tensor-core kernel: ``dX = dZ W^T`` (dZ is b x m, W n x m).  bf16 only."""
+    b, m = dZ.shape
+    n = W.shape[0]
+    dX = alloc_matrix(b, n, dZ.dtype, dZ.device) if dX is None else dX
+    _check(_lib.pamm_linear_backward_input(_ptr(dZ), _ld(dZ), b, m, _ptr(W), _ld(W), n, _dt(dZ), _ptr(dX), _ld(dX),
+                                           _stream(stream)), "pamm_linear_backward_input")
+    return dX
 
 
 def contract(f, alpha, dY, k: int, Btilde=None, sort_products=None, workspace=None, stream=None):

@@ -134,3 +134,20 @@ def test_fused_forward_full_size(name):
     parity.record(f"{name} fused forward k={w.ks[0]}", rep)
     # every row block and column tile was written: no element of Z is left at its initial value
     assert torch.isfinite(Z.float()).all()
+
+
+@pytest.mark.parametrize("b,n,m", [(1111, 200, 392), (300, 72, 40), (129, 64, 264), (4133, 520, 264), (256, 1032, 776)])
+def test_input_gradient_product(b, n, m):
+    # dX = dZ W^T (Algorithm 3) through the forward kernel with W as the operand whose contraction index is contiguous;
+    # the oracle's plain product of dZ with the transposed weight is the definition
+    dZ, _ = synth.random_case(b, m, 8, "bf16", seed=b + m)
+    W = make_weight(n, m, seed=n)
+    dX = pamm.linear_backward_input(parity.to_device(dZ), parity.to_device(W))
+    Wt = np.ascontiguousarray(W.T)
+    ref = orc.linear_forward(dZ, Wt)
+    rep = parity.Report(b=b, k=0)
+    parity.check_elementwise("dX", parity.to_f64(dX), ref, z_bound(dZ, Wt, ref), rep)
+    assert pamm.last_device_status() == pamm.OK
+    with pytest.raises(pamm.PammError) as e:
+        pamm.linear_backward_input(parity.to_device(dZ).float(), parity.to_device(W).float())
+    assert e.value.code == pamm.ERR_UNSUPPORTED
