@@ -534,3 +534,36 @@ def test_read_probes_visit_every_row_once():
     bad[17] = 3001
     pamm.probe_read(pamm.PROBE_ROWS, data, order=bad)
     assert pamm.last_device_status() == pamm.ERR_BAD_INDEX
+
+
+def test_calls_from_a_thread_that_has_not_touched_cuda_yet():
+    # a framework's worker thread (autograd's, a data loader's) may make its first CUDA call inside the library,
+    # and that call may start with a tensor-map encoding, which needs a current context
+    import threading
+    X, dY = synth.random_case(512, 256, 384, "bf16", seed=77)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, 32, 3)
+    Bt = pamm.contract(f, alpha, dYd, 32)
+    dW_main = pamm.weight_grad(C, Bt)
+    dX_main = pamm.linear_backward_input(dYd, parity.to_device(synth.f32_to_bf16_bits(np.ones((256, 384), np.float32))))
+    Wd = parity.to_device(synth.f32_to_bf16_bits(np.ones((256, 384), np.float32)))
+    dW_thr = torch.empty_like(dW_main)
+    dX_thr = torch.empty_like(dX_main)
+    torch.cuda.synchronize()
+    errors = []
+    stream = torch.cuda.current_stream()
+
+    def work():
+        try:
+            pamm.weight_grad(C, Bt, dW=dW_thr, stream=stream)
+            pamm.linear_backward_input(dYd, Wd, dX=dX_thr, stream=stream)
+        except Exception as e:      # noqa: BLE001
+            errors.append(e)
+
+    t = threading.Thread(target=work)
+    t.start()
+    t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    assert torch.equal(dW_thr, dW_main) and torch.equal(dX_thr.view(torch.int16), dX_main.view(torch.int16))
+    assert pamm.last_device_status() == pamm.OK
