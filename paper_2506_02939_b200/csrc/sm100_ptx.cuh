@@ -289,10 +289,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 inline EncodeTiledFn encode_tiled_fn() {
     // The driver call needs a current context.  A thread that has made no context-binding runtime call yet
     // (a framework's worker thread whose first library call goes straight to an encoding) has none:
-    // cudaFree(0) binds the device's primary context to the thread, once.
+    // cudaSetDevice on the thread's current device binds that device's primary context to the thread
+    // (and, unlike an allocation call, is harmless while a stream is being captured).
     static thread_local bool context_bound = false;
     if (!context_bound) {
-        cudaFree(0);
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaSetDevice(dev);
         context_bound = true;
     }
     static EncodeTiledFn fn = nullptr;
