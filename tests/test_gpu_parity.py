@@ -513,6 +513,44 @@ def test_a_whole_step_can_be_captured_in_a_cuda_graph():
         assert torch.equal(got, ref)
 
 
+def test_a_bf16_layer_with_many_generators_can_be_captured_in_a_cuda_graph():
+    # the kernels on pairs of CTAs (cluster launches) and the product over the bf16 planes, inside a graph
+    b, n, m, k = 2048, 512, 768, 256
+    X, dY = synth.random_case(b, n, m, "bf16", seed=82, centres=64, dy_scale=1e-3)
+    Xd, dYd = parity.to_device(X), parity.to_device(dY)
+    W = parity.to_device(synth.f32_to_bf16_bits(np.random.default_rng(3).standard_normal((n, m)).astype(np.float32) / 16))
+    sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, pamm.BF16)
+    Z, idx, C, invn, f, alpha = pamm.linear_forward(Xd, W, k, 5, sort_products=sp)
+    Bt = pamm.alloc_matrix(k, m, torch.float32)
+    dW = pamm.alloc_matrix(n, m, torch.float32)
+    dX = pamm.alloc_matrix(b, n, torch.bfloat16)
+    ws = pamm.alloc_workspace(pamm.WS_CONTRACT, b, n, m, k, pamm.BF16)
+
+    def step(stream=None):
+        pamm.linear_forward(Xd, W, k, 5, Z=Z, idx_out=idx, C=C, c_invnorm=invn, f=f, alpha=alpha, sort_products=sp, stream=stream)
+        pamm.contract_weight_grad(C, f, alpha, dYd, Btilde=Bt, dW=dW, sort_products=sp, workspace=ws, stream=stream)
+        pamm.linear_backward_input(dYd, W, dX=dX, stream=stream)
+
+    step()
+    torch.cuda.synchronize()
+    outs = (Z.view(torch.int16), f, alpha, Bt, dW, dX.view(torch.int16))
+    want = [t.clone() for t in outs]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step(torch.cuda.current_stream())
+    for t in outs:
+        t.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert pamm.last_device_status() == pamm.OK
+    for got, ref in zip(outs, want):
+        assert torch.equal(got, ref)
+
+
 def test_read_probes_visit_every_row_once():
     # no arithmetic of the method: the checksums only show that the probes read what they are timed for
     g = torch.Generator(device="cuda").manual_seed(5)
