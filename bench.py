@@ -488,7 +488,7 @@ def run_cuda(args):
     flops = 2.0 * b * k * n
     if w.dtype == "bf16" and t_compress > t_contract and flops / ab["compress"] > peak_tf * 1e12 / (peak * 1e9):
         tf = flops / t_compress / 1e12
-        roofline = {"bound": "tensor", "kernel": "compress_umma_kernel (scoring X C^T + argmax)", "achieved": tf, "peak": peak_tf,
+        roofline = {"bound": "tensor", "kernel": "compress_pair_kernel (scoring X C^T + argmax on pairs of CTAs)", "achieved": tf, "peak": peak_tf,
                     "peak_source": f"of {peak_kind} (sustained bf16)", "unit": "TFLOP/s", "frac": tf / peak_tf, "traffic": None,
                     "algorithmic_flops": flops, "samples": st_k["compress"]["count"]}
     else:
