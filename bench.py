@@ -452,6 +452,9 @@ def run_cuda(args):
     peak, peak_tf, peak_kind = measured_peaks()
     dw_e = 2 if args.dw_dtype == "bf16" else 4
     ab = algorithmic_bytes(b, n, m, k, e, dw_e)
+    # rows whose alpha is zero are left out of the contraction's sorted order and never read
+    rows_read = int((alpha != 0).sum().item())
+    ab["contract"] = rows_read * m * e + 8 * b
     st_f, st_b = stats(fwd), stats(bwd)
     st_k = {"compress": stats(kern[pamm.PROF_COMPRESS]), "contract_main": stats(kern[pamm.PROF_CONTRACT]),
             "weight_grad": stats(kern[pamm.PROF_WEIGHT_GRAD])}
@@ -537,6 +540,7 @@ def run_cuda(args):
         "clocks": clocks,
         "stages": stages,
         "read_ceiling": read_ceiling,
+        "rows_with_nonzero_alpha": rows_read,
         "memory_saved": saved,
     }
     print(json.dumps(line), flush=True)

@@ -126,7 +126,9 @@ pamm_status pamm_select_generators(const void* X, int64_t ldx, int64_t b, int64_
  *   alpha  b fp32
  *   workspace  NULL, or pamm_workspace_bytes(PAMM_WS_COMPRESS, ...) bytes that receive
  *          the "sort products": how many rows of every block of rows chose each
- *          generator, counted on the fly by the pass.  They are an optional by-product
+ *          generator, counted on the fly by the pass over the rows whose alpha is not
+ *          zero (a row with alpha = 0 adds nothing to B~ and the backward pass leaves it
+ *          out of its sorted order, so dY of such a row is never read).  They are an optional by-product
  *          for the backward pass (pamm_contract, pamm_contract_weight_grad), which then
  *          skips its own counting launch; they must be kept next to f until then and
  *          are valid only for this f on a device with the same number of SMs.  With
@@ -208,6 +210,8 @@ pamm_status pamm_compress_projections(const void* X, int64_t ldx, int64_t b, int
  * Step 3 -- contract (Section 3.2 "Approximate Matrix Multiplication";
  * Algorithm 1, ApproxMM: the alpha-scaling of B and the index_add into B~):
  *   B~[j,:] = sum over {i : f_i = j} of alpha_i * dY[i,:]      (k x m, fp32)
+ * Rows with alpha_i = 0 (dropped by the neighbourhood condition, all-zero rows) are skipped:
+ * their dY rows are not read, so a non-finite value there does not reach B~.
  * B' is never materialised.  dY is read once; rows are grouped by f with a
  * stable counting sort, summed in fp32 in ascending row order inside fixed-size
  * chunks, and chunk sums are added in ascending order -- no floating-point

@@ -245,8 +245,9 @@ compress_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                 if (!ok) break;
                 if (row < r1) {
                     store_index(out.f, out.f_type, (int64_t)g * out.out_stride + row, j_best);
-                    out.alpha[(int64_t)g * out.out_stride + row] = s_best * s_inv2[g * k + j_best];
-                    atomicAdd(&s_hist[g * k + j_best], 1);
+                    const float a = s_best * s_inv2[g * k + j_best];
+                    out.alpha[(int64_t)g * out.out_stride + row] = a;
+                    if (a != 0.f) atomicAdd(&s_hist[g * k + j_best], 1);     // a row with alpha = 0 takes no part in the backward pass
                 }
             }
         }

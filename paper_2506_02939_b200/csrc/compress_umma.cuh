@@ -28,9 +28,9 @@
 // Several independent generator sets ("groups": one compression per projection,
 // Section 4) are served by the same pass: the chunks of all groups follow one
 // another, the running argmax restarts at every group, and every group gets its
-// own f and alpha.  The epilogue also counts, per CTA and group, how many rows
-// chose each generator (integer atomics in shared memory): the per-block histograms
-// the backward pass's counting sort starts from.
+// own f and alpha.  The epilogue also counts, per CTA and group, how many rows with
+// alpha != 0 chose each generator (integer atomics in shared memory): the per-block
+// histograms the backward pass's counting sort starts from.
 #pragma once
 #include "pamm_common.cuh"
 #include "sm100_ptx.cuh"
@@ -426,7 +426,7 @@ compress_umma_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
                     }
                     store_index(out.f, out.f_type, (int64_t)g * out.out_stride + row, j_best);
                     out.alpha[(int64_t)g * out.out_stride + row] = a;
-                    atomicAdd(&s_hist[g * k + j_best], 1);
+                    if (a != 0.f) atomicAdd(&s_hist[g * k + j_best], 1);     // a row with alpha = 0 takes no part in the backward pass
                 }
                 if (EPS) {
                     __syncwarp();

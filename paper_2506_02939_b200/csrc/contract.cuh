@@ -61,9 +61,26 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
     return w;
 }
 
+// The key a row is sorted by: its generator f_i, or -1 for a row that takes no part -- one whose
+// alpha_i is zero (dropped by the neighbourhood condition, an all-zero row, a row orthogonal to its
+// generator: it adds nothing to B~ and is not read at all) or whose f_i is out of range (reported).
+// Every producer of the per-block counts uses the same rule.
+__device__ __forceinline__ int32_t sort_key(const void* f, int f_type, const float* alpha, int64_t i, int k) {
+    const int32_t j = load_index(f, f_type, i);
+    if (j < 0 || j >= k) {
+        raise_status(DEV_BAD_INDEX);
+        return -1;
+    }
+    return alpha[i] != 0.f ? j : -1;
+}
+
+// The rows of the sorted order are cut into `ranges` equal contiguous ranges (one CTA of the main
+// pass each); how many rows there are is known on the device only (rows with alpha = 0 are left out).
+__device__ __forceinline__ int range_rows(int32_t total, int ranges) { return max(1, (total + ranges - 1) / ranges); }
+
 __global__ void __launch_bounds__(SORT_BLK)
-contract_hist_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block,
-                     int32_t* __restrict__ hist) {
+contract_hist_kernel(const void* __restrict__ f, int f_type, const float* __restrict__ alpha, int64_t b, int k,
+                     int rows_per_block, int32_t* __restrict__ hist) {
     extern __shared__ int32_t s_hist[];
     for (int j = threadIdx.x; j < k; j += SORT_BLK) s_hist[j] = 0;
     grid_dependency_wait();     // f may come from the kernel before
@@ -72,9 +89,8 @@ contract_hist_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, i
     const int64_t i0 = (int64_t)blockIdx.x * rows_per_block;
     const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
     for (int64_t i = i0 + threadIdx.x; i < i1; i += SORT_BLK) {
-        const int32_t j = load_index(f, f_type, i);
-        if (j >= 0 && j < k) atomicAdd(&s_hist[j], 1);
-        else raise_status(DEV_BAD_INDEX);
+        const int32_t j = sort_key(f, f_type, alpha, i, k);
+        if (j >= 0) atomicAdd(&s_hist[j], 1);
     }
     __syncthreads();
     int32_t* out = hist + (int64_t)blockIdx.x * k;
@@ -201,9 +217,9 @@ inline int scatter_table_warps(int64_t rows_per_block, int64_t k) {
 
 // Stable scatter of one block's rows, given the scanned tables.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block, int tbl_warps,
-                        const int32_t* __restrict__ hist, const int32_t* __restrict__ seg_start,
-                        int32_t* __restrict__ perm) {
+contract_scatter_kernel(const void* __restrict__ f, int f_type, const float* __restrict__ alpha, int64_t b, int k,
+                        int rows_per_block, int tbl_warps, const int32_t* __restrict__ hist,
+                        const int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block, then the count table
     int32_t* s_tbl = tbl_warps ? s_next + k : nullptr;
     const int tid = threadIdx.x;
@@ -216,10 +232,7 @@ contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k
     for (int64_t c0 = i0; c0 < i1; c0 += SORT_BLK) {
         const int64_t i = c0 + tid;
         int32_t key = -1;
-        if (i < i1) {
-            key = load_index(f, f_type, i);
-            if (key < 0 || key >= k) key = -1;
-        }
+        if (i < i1) key = sort_key(f, f_type, alpha, i, k);
         scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), k, s_next, s_tbl, perm, b);
     }
 }
@@ -234,9 +247,9 @@ contract_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k
 // threads: with W = the chunk's width rounded up to a power of two, the SORT_BLK
 // / W thread groups each take every (SORT_BLK / W)-th histogram row.
 __global__ void __launch_bounds__(SORT_BLK)
-contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, int k, int rows_per_block, int tbl_warps,
-                             const int32_t* __restrict__ hist, int nb, int32_t* __restrict__ seg_start,
-                             int32_t* __restrict__ perm) {
+contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, const float* __restrict__ alpha, int64_t b, int k,
+                             int rows_per_block, int tbl_warps, const int32_t* __restrict__ hist, int nb,
+                             int32_t* __restrict__ seg_start, int32_t* __restrict__ perm) {
     extern __shared__ int32_t s_next[];    // next free slot of every segment for this block, then the count table
     int32_t* s_tbl = tbl_warps ? s_next + k : nullptr;
     __shared__ int32_t s_part[2][SORT_BLK];   // per-thread partial (total, before) of the column sums
@@ -249,7 +262,7 @@ contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, 
     const int64_t i0 = (int64_t)me * rows_per_block;
     const int64_t i1 = min(b, i0 + (int64_t)rows_per_block);
     // the keys of the first chunk travel while the column sums are formed
-    int32_t first_key = i0 + tid < i1 ? load_index(f, f_type, i0 + tid) : -1;
+    const int32_t first_key = i0 + tid < i1 ? sort_key(f, f_type, alpha, i0 + tid, k) : -1;
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < k; j0 += SORT_BLK) {
@@ -323,10 +336,7 @@ contract_scan_scatter_kernel(const void* __restrict__ f, int f_type, int64_t b, 
     for (int64_t c0 = i0; c0 < i1; c0 += SORT_BLK) {
         const int64_t i = c0 + tid;
         int32_t key = -1;
-        if (i < i1) {
-            key = c0 == i0 ? first_key : load_index(f, f_type, i);
-            if (key < 0 || key >= k) key = -1;
-        }
+        if (i < i1) key = c0 == i0 ? first_key : sort_key(f, f_type, alpha, i, k);
         scatter_chunk(key, i, (int)min((int64_t)SORT_BLK, i1 - c0), k, s_next, s_tbl, perm, b);
     }
 }
@@ -361,7 +371,7 @@ template <typename T>
 __global__ void __launch_bounds__(CT_MAX_THREADS)
 contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, int64_t ldy, int64_t b, int64_t m,
                      int k, const int32_t* __restrict__ seg_start, const int32_t* __restrict__ perm,
-                     int rows_per_cta, float* __restrict__ partials, int64_t m_pad,
+                     int ranges, float* __restrict__ partials, int64_t m_pad,
                      float* __restrict__ Bt, int64_t ldb) {
     constexpr int V = Vec16<T>::N;
     __shared__ int32_t s_row[CT_TILE];
@@ -370,6 +380,7 @@ contract_main_kernel(const float* __restrict__ alpha, const T* __restrict__ dY, 
     grid_dependency_wait();
     grid_launch_dependents();
     const int32_t total = (int32_t)min((int64_t)max(seg_start[k], 0), b);
+    const int rows_per_cta = range_rows(total, ranges);
     const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
     const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
     if (r_begin >= r_end) return;
@@ -463,7 +474,7 @@ constexpr int RED_THREADS = 256;
 // converted by every CTA that needs them.
 __global__ void __launch_bounds__(RED_THREADS)
 contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k, int64_t b,
-                       const int32_t* __restrict__ seg_start, int rows_per_cta,
+                       const int32_t* __restrict__ seg_start, int ranges,
                        float* __restrict__ Bt, int64_t ldb, uint16_t* __restrict__ planes, int64_t plane_ld) {
     const int64_t mv = m_pad / 4;
     const int64_t idx = (int64_t)blockIdx.x * RED_THREADS + threadIdx.x;
@@ -477,6 +488,7 @@ contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_
     float* out = Bt + (int64_t)j * ldb + col;
     bool written = false;      // the main pass wrote this row itself
     if (s1 > s0) {
+        const int rows_per_cta = range_rows((int32_t)min((int64_t)max(seg_start[k], 0), b), ranges);
         const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;
         if (c_lo == c_hi) {
             if (!planes) return;

@@ -2,7 +2,8 @@
 // B~[j,:] = sum_{i: f_i = j} alpha_i * dY[i,:] over the rows sorted by f, with the
 // rows of dY staged through shared memory by bulk asynchronous copies.
 //
-// The sorted rows are cut into equal contiguous ranges, one CTA per range, two
+// The sorted rows (those with alpha != 0: the others add nothing and are never read) are cut
+// into equal contiguous ranges, one CTA per range, two
 // CTAs per SM in a single balanced wave (two independent pipelines per SM hide
 // each other's waits; measured 17% faster than one CTA with twice the ring).
 // Inside a CTA:
@@ -74,7 +75,7 @@ template <typename T, int VPT, int RPS>
 __global__ void __launch_bounds__(CS_MAX_CONSUMERS + 32, CS_CTAS_PER_SM)
 contract_stream_kernel(const void* __restrict__ f, int f_type, const float* __restrict__ alpha, const T* __restrict__ dY,
                        int64_t ldy, int64_t b, int64_t m, int k, const int32_t* __restrict__ seg_start,
-                       const int32_t* __restrict__ perm, int rows_per_cta, int slots, int row_pitch,
+                       const int32_t* __restrict__ perm, int ranges, int slots, int row_pitch,
                        uint32_t bulk_bytes, float* __restrict__ partials, int64_t m_pad,
                        float* __restrict__ Bt, int64_t ldb) {
     constexpr int V = Vec16<T>::N;
@@ -102,7 +103,8 @@ contract_stream_kernel(const void* __restrict__ f, int f_type, const float* __re
     grid_dependency_wait();       // seg_start and perm come from the kernel before
     grid_launch_dependents();
 
-    const int32_t total = (int32_t)min((int64_t)max(seg_start[k], 0), b);     // = b unless some f_i were out of range
+    const int32_t total = (int32_t)min((int64_t)max(seg_start[k], 0), b);     // the rows with alpha != 0
+    const int rows_per_cta = range_rows(total, ranges);
     const int32_t r_begin = (int32_t)min((int64_t)c * rows_per_cta, (int64_t)total);
     const int32_t r_end = (int32_t)min((int64_t)r_begin + rows_per_cta, (int64_t)total);
     const int nrows = r_end - r_begin;

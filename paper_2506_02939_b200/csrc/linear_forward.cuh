@@ -158,8 +158,9 @@ __device__ __forceinline__ void lf_finish_scores(const LinearForwardOut& out, in
     const int64_t p0 = out.hist ? (rb * LF_TILE_M) / out.rows_per_block : 0;
     if (row < b) {
         store_index(out.f, out.f_type, row, j_best);
-        out.alpha[row] = s_best * s_inv2[j_best];
-        if (out.hist) atomicAdd(&s_hist[(int)(row / out.rows_per_block - p0) * k + j_best], 1);
+        const float a = s_best * s_inv2[j_best];
+        out.alpha[row] = a;
+        if (out.hist && a != 0.f) atomicAdd(&s_hist[(int)(row / out.rows_per_block - p0) * k + j_best], 1);
     }
     ptx::named_barrier(1, 128);
     if (out.hist) {

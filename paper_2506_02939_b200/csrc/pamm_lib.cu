@@ -229,8 +229,8 @@ constexpr int64_t FUSED_SCAN_LIMIT = 1ll << 24;
 
 // The counting sort of the rows by f.  `products` (the per-block histograms the compress
 // pass left behind) saves the histogram launch.
-pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const int32_t* products, const ContractWs& w,
-                        cudaStream_t st) {
+pamm_status launch_sort(const void* f, int f_type, const float* alpha, int64_t b, int64_t k, const int32_t* products,
+                        const ContractWs& w, cudaStream_t st) {
     if (k <= SK_MAX_K) products = nullptr;     // the forward pass for so few generators leaves no counts
     const size_t hsmem = (size_t)k * 4;
     const int rpb = (int)w.rows_per_block;
@@ -248,14 +248,14 @@ pamm_status launch_sort(const void* f, int f_type, int64_t b, int64_t k, const i
         if (cudaMemcpyAsync(w.hist, products, (size_t)w.nb * k * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
             return PAMM_ERR_CUDA;
     } else {
-        launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, b, (int)k, rpb, w.hist);
+        launch(contract_hist_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), hsmem, st, true, f, f_type, alpha, b, (int)k, rpb, w.hist);
     }
     if (fused_scan) {
-        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, b, (int)k, rpb,
-               tbl_warps, hist, (int)w.nb, w.seg_start, w.perm);
+        launch(contract_scan_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, alpha, b, (int)k,
+               rpb, tbl_warps, hist, (int)w.nb, w.seg_start, w.perm);
     } else {
         launch(contract_scan_kernel, dim3(1), dim3(SCAN_THREADS), 0, st, true, w.hist, (int)w.nb, (int)k, w.seg_start);
-        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, b, (int)k, rpb,
+        launch(contract_scatter_kernel, dim3((unsigned)w.nb), dim3(SORT_BLK), ssmem, st, true, f, f_type, alpha, b, (int)k, rpb,
                tbl_warps, (const int32_t*)w.hist, (const int32_t*)w.seg_start, w.perm);
     }
     return launch_status();
@@ -267,7 +267,7 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
                             cudaStream_t st, bool with_planes = false) {
     constexpr int V = Vec16<T>::N;
     uint16_t* planes = with_planes ? w.planes : nullptr;     // B~ also as bf16 hi / lo, for the product that follows
-    pamm_status s = launch_sort(f, f_type, b, k, products, w, st);
+    pamm_status s = launch_sort(f, f_type, alpha, b, k, products, w, st);
     if (s != PAMM_OK) return s;
     if (contract_stream_supported(m, sizeof(T))) {
         // one balanced wave, two CTAs per SM: rows of dY stream through a shared-memory ring
@@ -283,12 +283,12 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
         if (!ensure_dynamic_smem((const void*)kern, p.smem_bytes)) return PAMM_ERR_CUDA;
         prof_begin(PAMM_PROF_CONTRACT, st);
         launch(kern, dim3((unsigned)ranges), dim3(p.consumers + 32), p.smem_bytes, st, true, f, f_type, alpha, (const T*)dY,
-               ldy, b, m, (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, p.slots,
+               ldy, b, m, (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)ranges, p.slots,
                p.row_pitch, p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
         prof_end(PAMM_PROF_CONTRACT, st);
         const int64_t items = k * (w.m_pad / 4);
         launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st,
-               true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb, planes, w.plane_ld);
+               true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)ranges, Bt, ldb, planes, w.plane_ld);
         return launch_status();
     }
     // very wide rows: column slabs, register staging
@@ -304,11 +304,11 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
     dim3 grid((unsigned)ranges, (unsigned)slabs);
     prof_begin(PAMM_PROF_CONTRACT, st);
     launch(contract_main_kernel<T>, grid, dim3(threads), 0, st, true, alpha, (const T*)dY, ldy, b, m, (int)k,
-           (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)rows_per_cta, w.partials, w.m_pad, Bt, ldb);
+           (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)ranges, w.partials, w.m_pad, Bt, ldb);
     prof_end(PAMM_PROF_CONTRACT, st);
     const int64_t items = k * (w.m_pad / 4);
     launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st, true,
-           (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)rows_per_cta, Bt, ldb, planes, w.plane_ld);
+           (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)ranges, Bt, ldb, planes, w.plane_ld);
     return launch_status();
 }
 
@@ -490,7 +490,7 @@ pamm_status do_compress(const void* X, int64_t ldx, int64_t b, int64_t n, pamm_d
         if (s != PAMM_OK) return s;
         if (products)
             launch(contract_hist_kernel, dim3((unsigned)nblk), dim3(SORT_BLK), (size_t)k * 4, st, true, (const void*)fg,
-                   (int)f_type, b, (int)k, (int)rpb, products + (size_t)g * (sort_products_bytes(b, k) / 4));
+                   (int)f_type, (const float*)ag, b, (int)k, (int)rpb, products + (size_t)g * (sort_products_bytes(b, k) / 4));
     }
     return launch_status();
 }
