@@ -605,3 +605,32 @@ def test_calls_from_a_thread_that_has_not_touched_cuda_yet():
     assert not errors, errors
     assert torch.equal(dW_thr, dW_main) and torch.equal(dX_thr.view(torch.int16), dX_main.view(torch.int16))
     assert pamm.last_device_status() == pamm.OK
+
+
+def test_rows_with_zero_alpha_are_never_read():
+    # a row with alpha = 0 adds nothing to B~ (Section 3.2: B~_j is a sum of alpha_i B_i): the backward pass leaves it
+    # out of its sorted order, so whatever its row of dY holds -- here NaNs -- does not reach B~ or dW
+    b, n, m, k = 3000, 256, 520, 32
+    X, dY = synth.random_case(b, n, m, "bf16", seed=91, centres=20)
+    zero_rows = np.arange(7, b, 13)
+    X = X.copy()
+    X[zero_rows] = 0                                  # all-zero rows: S = 0, alpha = 0
+    poisoned = dY.copy()
+    poisoned[zero_rows] = 0x7FC0                      # bf16 NaN
+    cleaned = dY.copy()
+    cleaned[zero_rows] = 0
+    Xd = parity.to_device(X)
+    for with_products in (True, False):
+        sp = pamm.alloc_workspace(pamm.WS_COMPRESS, b, n, m, k, pamm.BF16) if with_products else None
+        idx, C, invn, f, alpha = pamm.compress_fused(Xd, k, 4, sort_products=sp)
+        assert torch.all(alpha[torch.from_numpy(zero_rows).cuda()] == 0)
+        Bt_p = pamm.alloc_matrix(k, m, torch.float32)
+        Bt_c = pamm.alloc_matrix(k, m, torch.float32)
+        dW_p = pamm.contract_weight_grad(C, f, alpha, parity.to_device(poisoned), Btilde=Bt_p, sort_products=sp)
+        dW_c = pamm.contract_weight_grad(C, f, alpha, parity.to_device(cleaned), Btilde=Bt_c, sort_products=sp)
+        assert pamm.last_device_status() == pamm.OK
+        assert torch.isfinite(Bt_p).all() and torch.isfinite(dW_p).all()
+        assert torch.equal(Bt_p, Bt_c) and torch.equal(dW_p, dW_c)
+    # and against the oracle on the cleaned input
+    for products in (False, True):
+        parity.run_and_compare(X, cleaned, k, seed=4, products=products)
