@@ -67,11 +67,12 @@ inline ContractWs contract_ws_layout(void* base, int64_t b, int64_t m, int64_t k
 // Every producer of the per-block counts uses the same rule.
 __device__ __forceinline__ int32_t sort_key(const void* f, int f_type, const float* alpha, int64_t i, int k) {
     const int32_t j = load_index(f, f_type, i);
+    const float a = alpha[i];            // both loads travel together
     if (j < 0 || j >= k) {
         raise_status(DEV_BAD_INDEX);
         return -1;
     }
-    return alpha[i] != 0.f ? j : -1;
+    return a != 0.f ? j : -1;
 }
 
 // The rows of the sorted order are cut into `ranges` equal contiguous ranges (one CTA of the main
