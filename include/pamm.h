@@ -211,7 +211,7 @@ pamm_status pamm_compress_projections(const void* X, int64_t ldx, int64_t b, int
  * Algorithm 1, ApproxMM: the alpha-scaling of B and the index_add into B~):
  *   B~[j,:] = sum over {i : f_i = j} of alpha_i * dY[i,:]      (k x m, fp32)
  * Rows with alpha_i = 0 (dropped by the neighbourhood condition, all-zero rows) are skipped:
- * their dY rows are not read, so a non-finite value there does not reach B~.
+ * a non-finite value in their dY rows does not reach B~ (with k > 8 those rows are not even read).
  * B' is never materialised.  dY is read once; rows are grouped by f with a
  * stable counting sort, summed in fp32 in ascending row order inside fixed-size
  * chunks, and chunk sums are added in ascending order -- no floating-point

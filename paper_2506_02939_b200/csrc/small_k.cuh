@@ -208,8 +208,9 @@ contract_small_kernel(const void* __restrict__ f, int f_type, const float* __res
                 if (blockIdx.y == 0) raise_status(DEV_BAD_INDEX);
                 j = -1;
             }
-            s_f[tid] = j;
-            s_a[tid] = alpha[t0 + tid];
+            const float a = alpha[t0 + tid];
+            s_f[tid] = a != 0.f ? j : -1;       // a row with alpha = 0 adds nothing: it matches no generator below
+            s_a[tid] = a;
         }
         __syncthreads();
         if (!active) continue;

@@ -634,3 +634,8 @@ def test_rows_with_zero_alpha_are_never_read():
     # and against the oracle on the cleaned input
     for products in (False, True):
         parity.run_and_compare(X, cleaned, k, seed=4, products=products)
+    # a handful of generators (the path without a sort): the same rule
+    idx, C, invn, f, alpha = pamm.compress_fused(Xd, 4, 4)
+    dW_p = pamm.contract_weight_grad(C, f, alpha, parity.to_device(poisoned))
+    dW_c = pamm.contract_weight_grad(C, f, alpha, parity.to_device(cleaned))
+    assert torch.isfinite(dW_p).all() and torch.equal(dW_p, dW_c)
