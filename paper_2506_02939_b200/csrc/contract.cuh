@@ -477,63 +477,63 @@ __global__ void __launch_bounds__(RED_THREADS)
 contract_reduce_kernel(const float* __restrict__ partials, int64_t m_pad, int64_t m, int k, int64_t b,
                        const int32_t* __restrict__ seg_start, int ranges,
                        float* __restrict__ Bt, int64_t ldb, uint16_t* __restrict__ planes, int64_t plane_ld) {
-    const int64_t mv = m_pad / 4;
-    const int64_t idx = (int64_t)blockIdx.x * RED_THREADS + threadIdx.x;
+    // grid: x over groups of four columns, y over the generators (no divisions; a CTA's threads share the segment's bounds)
+    const int64_t col = ((int64_t)blockIdx.x * RED_THREADS + threadIdx.x) * 4;
     grid_dependency_wait();
     grid_launch_dependents();
-    if (idx >= (int64_t)k * mv) return;
-    const int j = (int)(idx / mv);
-    const int64_t col = (idx % mv) * 4;
-    const int32_t s0 = (int32_t)min((int64_t)max(seg_start[j], 0), b), s1 = (int32_t)min((int64_t)max(seg_start[j + 1], 0), b);
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    float* out = Bt + (int64_t)j * ldb + col;
-    bool written = false;      // the main pass wrote this row itself
-    if (s1 > s0) {
-        const int rows_per_cta = range_rows((int32_t)min((int64_t)max(seg_start[k], 0), b), ranges);
-        const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;
-        if (c_lo == c_hi) {
-            if (!planes) return;
-            written = true;
-            if (col + 4 <= m) {
-                s = *reinterpret_cast<const float4*>(out);
+    if (col >= m_pad) return;
+    for (int j = blockIdx.y; j < k; j += gridDim.y) {
+        const int32_t s0 = (int32_t)min((int64_t)max(seg_start[j], 0), b), s1 = (int32_t)min((int64_t)max(seg_start[j + 1], 0), b);
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        float* out = Bt + (int64_t)j * ldb + col;
+        bool written = false;      // the main pass wrote this row itself
+        if (s1 > s0) {
+            const int rows_per_cta = range_rows((int32_t)min((int64_t)max(seg_start[k], 0), b), ranges);
+            const int c_lo = s0 / rows_per_cta, c_hi = (s1 - 1) / rows_per_cta;
+            if (c_lo == c_hi) {
+                if (!planes) continue;
+                written = true;
+                if (col + 4 <= m) {
+                    s = *reinterpret_cast<const float4*>(out);
+                } else {
+                    float v[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int e = 0; e < 4 && col + e < m; ++e) v[e] = out[e];
+                    s = make_float4(v[0], v[1], v[2], v[3]);
+                }
             } else {
-                float v[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int e = 0; e < 4 && col + e < m; ++e) v[e] = out[e];
-                s = make_float4(v[0], v[1], v[2], v[3]);
-            }
-        } else {
-            for (int c = c_lo; c <= c_hi; ++c) {
-                const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)(c + j) * m_pad + col);
-                s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+                for (int c = c_lo; c <= c_hi; ++c) {
+                    const float4 p = *reinterpret_cast<const float4*>(partials + (int64_t)(c + j) * m_pad + col);
+                    s.x += p.x; s.y += p.y; s.z += p.z; s.w += p.w;
+                }
             }
         }
-    }
-    if (!written) {
-        if (col + 4 <= m) {
-            *reinterpret_cast<float4*>(out) = s;
-        } else {
-            const float v[4] = {s.x, s.y, s.z, s.w};
-            for (int e = 0; e < 4 && col + e < m; ++e) out[e] = v[e];
+        if (!written) {
+            if (col + 4 <= m) {
+                *reinterpret_cast<float4*>(out) = s;
+            } else {
+                const float v[4] = {s.x, s.y, s.z, s.w};
+                for (int e = 0; e < 4 && col + e < m; ++e) out[e] = v[e];
+            }
         }
-    }
-    if (planes) {
-        const float x[4] = {s.x, s.y, s.z, s.w};
-        float h[4], l[4];
+        if (planes) {
+            const float x[4] = {s.x, s.y, s.z, s.w};
+            float h[4], l[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const bool in = col + e < m;
-            h[e] = in ? __bfloat162float(__float2bfloat16_rn(x[e])) : 0.f;
-            l[e] = in ? x[e] - h[e] : 0.f;
-        }
-        auto pack2 = [](float a, float c) {
-            __nv_bfloat162 t = __floats2bfloat162_rn(a, c);     // .x = first argument = low 16 bits
-            return *reinterpret_cast<uint32_t*>(&t);
-        };
-        uint16_t* hi = planes + (int64_t)j * plane_ld + col;      // col % 4 == 0 and plane_ld % 8 == 0: 8-byte aligned
-        uint16_t* lo = hi + (int64_t)k * plane_ld;
-        if (col + 4 <= plane_ld) {
-            *reinterpret_cast<uint2*>(hi) = make_uint2(pack2(h[0], h[1]), pack2(h[2], h[3]));
-            *reinterpret_cast<uint2*>(lo) = make_uint2(pack2(l[0], l[1]), pack2(l[2], l[3]));
+            for (int e = 0; e < 4; ++e) {
+                const bool in = col + e < m;
+                h[e] = in ? __bfloat162float(__float2bfloat16_rn(x[e])) : 0.f;
+                l[e] = in ? x[e] - h[e] : 0.f;
+            }
+            auto pack2 = [](float a, float c) {
+                __nv_bfloat162 t = __floats2bfloat162_rn(a, c);     // .x = first argument = low 16 bits
+                return *reinterpret_cast<uint32_t*>(&t);
+            };
+            uint16_t* hi = planes + (int64_t)j * plane_ld + col;      // col % 4 == 0 and plane_ld % 8 == 0: 8-byte aligned
+            uint16_t* lo = hi + (int64_t)k * plane_ld;
+            if (col + 4 <= plane_ld) {
+                *reinterpret_cast<uint2*>(hi) = make_uint2(pack2(h[0], h[1]), pack2(h[2], h[3]));
+                *reinterpret_cast<uint2*>(lo) = make_uint2(pack2(l[0], l[1]), pack2(l[2], l[3]));
+            }
         }
     }
 }

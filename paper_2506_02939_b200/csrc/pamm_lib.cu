@@ -286,8 +286,7 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
                ldy, b, m, (int)k, (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)ranges, p.slots,
                p.row_pitch, p.bulk_bytes, w.partials, w.m_pad, Bt, ldb);
         prof_end(PAMM_PROF_CONTRACT, st);
-        const int64_t items = k * (w.m_pad / 4);
-        launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st,
+        launch(contract_reduce_kernel, dim3((unsigned)((w.m_pad / 4 + RED_THREADS - 1) / RED_THREADS), (unsigned)std::min<int64_t>(k, 65535)), dim3(RED_THREADS), 0, st,
                true, (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)ranges, Bt, ldb, planes, w.plane_ld);
         return launch_status();
     }
@@ -306,8 +305,7 @@ pamm_status launch_contract(const void* f, int f_type, const float* alpha, const
     launch(contract_main_kernel<T>, grid, dim3(threads), 0, st, true, alpha, (const T*)dY, ldy, b, m, (int)k,
            (const int32_t*)w.seg_start, (const int32_t*)w.perm, (int)ranges, w.partials, w.m_pad, Bt, ldb);
     prof_end(PAMM_PROF_CONTRACT, st);
-    const int64_t items = k * (w.m_pad / 4);
-    launch(contract_reduce_kernel, dim3((unsigned)((items + RED_THREADS - 1) / RED_THREADS)), dim3(RED_THREADS), 0, st, true,
+    launch(contract_reduce_kernel, dim3((unsigned)((w.m_pad / 4 + RED_THREADS - 1) / RED_THREADS), (unsigned)std::min<int64_t>(k, 65535)), dim3(RED_THREADS), 0, st, true,
            (const float*)w.partials, w.m_pad, m, (int)k, b, (const int32_t*)w.seg_start, (int)ranges, Bt, ldb, planes, w.plane_ld);
     return launch_status();
 }
